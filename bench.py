@@ -1,0 +1,359 @@
+#!/usr/bin/env python
+"""Benchmark of the gated delta rule hot path on B200: decode state-GB/s and prefill tokens/s.
+
+One step = one decode call on the B=64 configuration (64 sequences x 32 v-heads, a 128 MiB fp32
+state pool updated in place) followed by one chunked prefill call on the packed variable-length
+configuration (4 sequences, 7680 tokens).  Both are timed separately with CUDA events on the
+launching stream, after an L2 flush.  The headline `value` is decode state-GB/s; the prefill
+leg's tokens/s and roofline are reported in the same JSON line under "prefill".
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+With N > 1 (launched by torch.distributed.run) every rank runs the same per-GPU workload on its
+own GPU (independent sequences, no data-path collective: weak scaling); the timed region is
+bracketed by a barrier and the per-step times are the max over ranks.
+`--impl reference` times the fp64 CPU oracle on the host cores on the same metric.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2607_17979_b200 import inputs as I  # noqa: E402
+
+DECODE_CFG, PREFILL_CFG = 1, 3
+TILE_BYTES = 128 * 128 * 4
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures
+# (profiles/); None until a capture of that kernel exists.
+NCU_TRAFFIC_BYTES = {"decode": None, "prefill": None}
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def decode_bytes(B, Hqk, Hv, with_idx):
+    """Algorithmic bytes of one decode call: state read + written, q, k, v, o, g, beta (+ slots)."""
+    state = 2 * B * Hv * TILE_BYTES
+    other = B * (2 * Hqk * 128 * 2 + 2 * Hv * 128 * 2 + 2 * Hv * 4 + (4 if with_idx else 0))
+    return state, state + other
+
+
+def prefill_bytes_flops(T, N, Hqk, Hv, with_init):
+    """Algorithmic bytes / flops of one prefill call (triangular products at half, Gram products
+    once per q/k head): 24832 B and 4194304 flop per token at Hqk=16, Hv=32."""
+    per_tok = 2 * Hqk * 128 * 2 + 2 * Hv * 128 * 2 + 2 * Hv * 4
+    nbytes = T * per_tok + N * Hv * TILE_BYTES * (2 if with_init else 1) + 4 * (N + 1)
+    flops = T * (Hqk * 16384 + Hv * 122880)
+    return nbytes, flops
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-i", str(self.gpu), "-lms", "50"], stdout=open(self.path, "w"),
+                stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def oracle_sample(dec, pre, decode_reps=5):
+    """Time the fp64 oracle, as it stands, on the host cores: the whole decode configuration
+    (`decode_reps` consecutive steps on its pool) and the whole prefill configuration once."""
+    import oracle
+    oracle.build()
+    cores = min(oracle.default_threads(), len(os.sched_getaffinity(0)))
+    pool = dec["state"].astype(np.float64)
+    t0 = time.perf_counter()
+    for _ in range(decode_reps):
+        oracle.decode(dec["q"], dec["k"], dec["v"], dec["g"], dec["beta"], pool, dec["slot_idx"],
+                      dec["scale"], n_threads=cores)
+    t_dec = (time.perf_counter() - t0) / decode_reps
+    t0 = time.perf_counter()
+    oracle.prefill(pre["q"], pre["k"], pre["v"], pre["g"], pre["beta"], pre["cu_seqlens"], None, None,
+                   pre["scale"], n_threads=cores)
+    t_pre = time.perf_counter() - t0
+    state_bytes, _ = decode_bytes(dec["B"], dec["Hqk"], dec["Hv"], dec["slot_idx"] is not None)
+    return dict(cores=cores, decode_s=t_dec, decode_state_gbs=state_bytes / t_dec / 1e9,
+                prefill_s=t_pre, prefill_tokens=pre["T"], prefill_tok_s=pre["T"] / t_pre,
+                sample=(f"decode: the whole B={dec['B']} step, mean of {decode_reps} consecutive "
+                        f"steps ({t_dec * 1e3:.1f} ms each; state bytes counted as fp32); prefill: "
+                        f"the whole varlen batch ({pre['T']} tokens, {pre['Hv']} v-heads, "
+                        f"{t_pre:.2f} s)"))
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    dec = I.make_config(DECODE_CFG)
+    pre = I.make_config(PREFILL_CFG)
+    for _ in range(args.warmup):
+        r = oracle_sample(dec, pre)
+    times, gbs, last = [], [], None
+    for _ in range(args.steps):
+        last = oracle_sample(dec, pre)
+        times.append(last["decode_s"] + last["prefill_s"])
+        gbs.append(last["decode_state_gbs"])
+    dec_gbs = float(np.mean(gbs))
+    line = {
+        "impl": "reference", "metric": "gdn_decode_state_GBps", "value": dec_gbs, "unit": "GB/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * float(np.mean(times)), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "decode B=64 Hqk=16 Hv=32 d=128 (configs[1]) + prefill 4 seqs, 7680 "
+                               "tokens (configs[3]), fp64 oracle on host cores", "l2": "host run"},
+        "cpu_baseline": {"value": dec_gbs, "unit": "GB/s", "cores": last["cores"], "kind": "oracle",
+                         "sample": last["sample"]},
+        "prefill": {"metric": "gdn_prefill_tokens_per_s", "value": last["prefill_tok_s"],
+                    "unit": "tokens/s"},
+        "e2e": {"value": dec_gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2607_17979_b200 import api
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def bf16(bits):
+        return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+    def dev(x):
+        return None if x is None else torch.from_numpy(x).cuda()
+
+    # every rank owns its own sequences (different seeds): weak scaling, no exchange
+    dec = I.make_config(DECODE_CFG, trial=rank)
+    pre = I.make_config(PREFILL_CFG, trial=rank)
+    B, Hqk, Hv = dec["B"], dec["Hqk"], dec["Hv"]
+    T, N = pre["T"], pre["N"]
+
+    d_in = {n: (bf16(dec[n]) if n in "qkv" else dev(dec[n])) for n in ("q", "k", "v", "g", "beta")}
+    pool = dev(dec["state"])
+    d_o = torch.empty((B, Hv, 128), dtype=torch.bfloat16, device="cuda")
+    p_in = {n: (bf16(pre[n]) if n in "qkv" else dev(pre[n])) for n in ("q", "k", "v", "g", "beta")}
+    cu = dev(pre["cu_seqlens"])
+    p_final = torch.empty((N, Hv, 128, 128), dtype=torch.float32, device="cuda")
+    p_o = torch.empty((T, Hv, 128), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(max(api.gdn_prefill_workspace_bytes(T, N, Hqk, Hv), 256), dtype=torch.uint8,
+                     device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")       # 4x the 126 MB L2
+
+    # pinned host copies for the end-to-end leg
+    h_dec = {n: t.cpu().pin_memory() for n, t in d_in.items()}
+    h_do = torch.empty_like(d_o, device="cpu").pin_memory()
+    h_pre = {n: t.cpu().pin_memory() for n, t in p_in.items()}
+    h_cu = cu.cpu().pin_memory()
+    h_po = torch.empty_like(p_o, device="cpu").pin_memory()
+
+    def decode_call():
+        api.gdn_decode(d_in["q"], d_in["k"], d_in["v"], d_in["g"], d_in["beta"], pool, None, d_o,
+                       dec["scale"], status)
+
+    def prefill_call():
+        api.gdn_prefill(p_in["q"], p_in["k"], p_in["v"], p_in["g"], p_in["beta"], cu, None, p_final,
+                        None, p_o, pre["scale"], ws, max_seqlen_hint=max(pre["seq_lens"]),
+                        dev_status=status)
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    def step(timed):
+        flush.zero_()
+        e0, e1, e2, e3 = ev(), ev(), ev(), ev()
+        e0.record(); decode_call(); e1.record()
+        flush.zero_()
+        e2.record(); prefill_call(); e3.record()
+        if timed is not None:
+            timed.append((e0, e1, e2, e3))
+
+    def e2e_step(timed):
+        flush.zero_()
+        e0, e1, e2, e3 = ev(), ev(), ev(), ev()
+        e0.record()
+        for n in d_in:
+            d_in[n].copy_(h_dec[n], non_blocking=True)
+        decode_call()
+        h_do.copy_(d_o, non_blocking=True)
+        e1.record()
+        flush.zero_()
+        e2.record()
+        for n in p_in:
+            p_in[n].copy_(h_pre[n], non_blocking=True)
+        cu.copy_(h_cu, non_blocking=True)
+        prefill_call()
+        h_po.copy_(p_o, non_blocking=True)
+        e3.record()
+        if timed is not None:
+            timed.append((e0, e1, e2, e3))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed_region(fn):
+        for _ in range(args.warmup):
+            fn(None)
+        barrier()
+        evs = []
+        for _ in range(args.steps):
+            fn(evs)
+        barrier()
+        dec_ms = np.array([a.elapsed_time(b) for a, b, _, _ in evs])
+        pre_ms = np.array([c.elapsed_time(d) for _, _, c, d in evs])
+        t = torch.tensor([dec_ms.mean(), pre_ms.mean()], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t[0]), float(t[1])
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    dec_ms, pre_ms = timed_region(step)
+    clocks = sampler.stop() if rank == 0 else None
+    e2e_dec_ms, e2e_pre_ms = timed_region(e2e_step)
+    assert int(status.item()) == 0, "device status flagged during the benchmark"
+
+    if rank == 0:
+        pk, pk_kind = peaks()
+        state_b, dec_b = decode_bytes(B, Hqk, Hv, False)
+        pre_b, pre_f = prefill_bytes_flops(T, N, Hqk, Hv, False)
+        dec_gbs = world * state_b / (dec_ms * 1e-3) / 1e9
+        dec_ach = dec_b / (dec_ms * 1e-3) / 1e9
+        pre_tok = world * T / (pre_ms * 1e-3)
+        pre_ach = pre_b / (pre_ms * 1e-3) / 1e9
+        pre_roof_ms = max(pre_b / (pk["hbm_gbs"] * 1e9),
+                          pre_f / (pk["bf16_tflops_sustained"] * 1e12)) * 1e3
+        cpu = oracle_sample(dec, pre)
+        h2d = sum(t.numel() * t.element_size() for t in h_dec.values())
+        h2d_p = sum(t.numel() * t.element_size() for t in h_pre.values()) + h_cu.numel() * 4
+        line = {
+            "metric": "gdn_decode_state_GBps", "value": dec_gbs, "unit": "GB/s",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": dec_ms + pre_ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "step = gdn_decode B=64 Hqk=16 Hv=32 d=128, 128 MiB fp32 state "
+                                   "pool in place (configs[1]) + gdn_prefill 4 seqs "
+                                   "{512,1024,2048,4096} = 7680 tokens, chunk 64 (configs[3])",
+                       "per_gpu": True,
+                       "l2": "512 MiB buffer written before each timed call (L2 flush)",
+                       "decode_ms": dec_ms, "prefill_ms": pre_ms},
+            "roofline": {"kernel": "gdn decode", "bound": "hbm", "achieved": dec_ach,
+                         "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": dec_ach / pk["hbm_gbs"],
+                         "peak_kind": pk_kind, "frac_of_nominal_8TBps": dec_ach / 8000.0,
+                         "algorithmic_bytes": dec_b, "traffic": NCU_TRAFFIC_BYTES["decode"]},
+            "prefill": {"metric": "gdn_prefill_tokens_per_s", "value": pre_tok, "unit": "tokens/s",
+                        "ms": pre_ms, "dtype": "bf16 operands, f32 accumulate and state",
+                        "roofline": {"kernel": "gdn prefill (all launches of one call)",
+                                     "bound": "hbm", "achieved": pre_ach, "peak": pk["hbm_gbs"],
+                                     "unit": "GB/s", "frac": pre_ach / pk["hbm_gbs"],
+                                     "peak_kind": pk_kind, "roofline_ms": pre_roof_ms,
+                                     "frac_of_roofline_time": pre_roof_ms / pre_ms,
+                                     "algorithmic_bytes": pre_b, "algorithmic_flops": pre_f,
+                                     "traffic": NCU_TRAFFIC_BYTES["prefill"]},
+                        "e2e": {"value": world * T / (e2e_pre_ms * 1e-3), "unit": "tokens/s",
+                                "h2d_bytes_per_step": h2d_p,
+                                "d2h_bytes_per_step": h_po.numel() * 2},
+                        "cpu_baseline": {"value": cpu["prefill_tok_s"], "unit": "tokens/s"}},
+            "cpu_baseline": {"value": cpu["decode_state_gbs"], "unit": "GB/s", "cores": cpu["cores"],
+                             "kind": "oracle", "sample": cpu["sample"]},
+            "e2e": {"value": world * state_b / (e2e_dec_ms * 1e-3) / 1e9, "unit": "GB/s",
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": h_do.numel() * 2,
+                    "note": "q,k,v,g,beta from pinned host memory and o back each step; the state "
+                            "pool is the resident recurrent cache and stays in HBM"},
+            "gpu_launches": args.steps * api.LAUNCHES_PER_STEP,
+            "clocks": clocks,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,157 @@
+/*
+ * gdn.h - C ABI of the B200 (sm_100a) gated delta rule library.
+ *
+ * Operator (paper, appendix "Operator Background and Mathematical Definitions",
+ * subsection "Gated Delta Net", the gated delta rule):
+ *
+ *     S_t = S_{t-1} ( alpha_t ( I - beta_t k_t k_t^T ) ) + beta_t v_t k_t^T
+ *     o_t = scale * S_t q_t                  (the paper writes it with scale = 1)
+ *
+ * S is a dv x dk matrix state per (sequence, v-head); alpha_t = exp(g_t) is the
+ * log-domain ("natural-log") gate the same subsection describes.  The paper's
+ * two execution regimes are the two entry points: decode (a prior state plus
+ * one new token) and prefill (whole packed sequences, outputs plus final state,
+ * evaluated through chunked matrix operations).
+ *
+ * Conventions fixed by this library (the paper leaves them open):
+ *   - grouped heads: v-head hv uses q/k head  hv / (Hv / Hqk);  Hv % Hqk == 0.
+ *   - a state tile is row-major [dv][dk], dk contiguous, fp32.
+ *   - q, k, v, o are bf16 (raw 16-bit), g and beta fp32, all contiguous.
+ *   - only dk == dv == 128 and chunk == 64 are supported.
+ *
+ * Common rules for every call below
+ *   - Every pointer is DEVICE memory owned by the caller unless a comment says
+ *     "host".  The library allocates nothing and keeps no state between calls
+ *     except where an entry point's own comment says otherwise.
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*) and return
+ *     without synchronising.  No device data is read on the host.
+ *   - Return value: 0 = enqueued; negative = rejected before any launch and
+ *     nothing was written (see GDN_ERR_*).
+ *   - Problems only the device can see set bits in *dev_status (device int32,
+ *     may be NULL; bits are OR-ed in, never cleared by the library) and the
+ *     offending unit is skipped; the kernels never trap.
+ */
+#ifndef GDN_B200_H_
+#define GDN_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GDN_OK                 0
+#define GDN_ERR_NULL          -1  /* a required pointer is NULL                              */
+#define GDN_ERR_SIZE          -2  /* a negative size, or num_slots <= 0 with work to do       */
+#define GDN_ERR_SHAPE         -3  /* dk, dv != 128, chunk != 64, Hv % Hqk != 0, ...           */
+#define GDN_ERR_ALIGN         -4  /* q/k/v/o/state/workspace not 16-byte aligned              */
+#define GDN_ERR_WORKSPACE     -5  /* workspace_bytes smaller than the size query answers      */
+#define GDN_ERR_CUDA          -6  /* the CUDA runtime refused a launch or a set-up call       */
+#define GDN_ERR_LIMIT         -7  /* a size exceeds a fixed maximum stated by the entry point */
+
+#define GDN_DEV_BAD_SLOT       1  /* a slot index >= num_slots was skipped                    */
+#define GDN_DEV_BAD_CU_SEQLENS 2  /* cu_seqlens not non-decreasing from 0 to T; unit skipped   */
+#define GDN_DEV_TIMEOUT        4  /* a bounded wait inside a kernel gave up                   */
+
+/*
+ * gdn_decode - one token of the gated delta rule for each of B sequences
+ * (paper: "Decode receives a prior state and computes ... new recurrent
+ * updates"; here exactly one update per sequence per call).
+ *
+ * For entry i and v-head hv, with slot = slot_idx ? slot_idx[i] : i and the
+ * tile S = state_pool[slot][hv]:
+ *     S <- exp(g) S ;  u = S k ;  S <- S + beta (v - u) k^T ;  o = scale S q
+ * The tile is read once and written back in place; o is rounded to bf16.
+ *
+ *   q, k        bf16 [B][Hqk][dk]
+ *   v           bf16 [B][Hv][dv]
+ *   g, beta     fp32 [B][Hv]          g = ln(alpha)
+ *   state_pool  fp32 [num_slots][Hv][dv][dk], updated in place
+ *   slot_idx    int32 [B] or NULL.  A negative index is a padding entry: its
+ *               o rows are zero and no state is touched.  An index >=
+ *               num_slots does the same and sets GDN_DEV_BAD_SLOT.  Two
+ *               entries naming the same slot in one call race (undefined).
+ *   o           bf16 [B][Hv][dv], written
+ * B == 0 is a no-op that returns 0.
+ */
+int gdn_decode(const void* q, const void* k, const void* v,
+               const float* g, const float* beta,
+               float* state_pool, const int32_t* slot_idx, void* o,
+               int32_t B, int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv,
+               int32_t num_slots, float scale,
+               int32_t* dev_status, void* stream);
+
+/*
+ * gdn_prefill_workspace_bytes - device scratch gdn_prefill needs for a packed
+ * batch of at most T tokens in at most N sequences.  Returns 0 for shapes
+ * gdn_prefill would reject.
+ */
+size_t gdn_prefill_workspace_bytes(int32_t T, int32_t N, int32_t Hqk, int32_t Hv,
+                                   int32_t dk, int32_t dv, int32_t chunk);
+
+/*
+ * gdn_prefill - the same recurrence over N packed variable-length sequences
+ * (paper: "Prefill evaluates a whole sequence and returns both outputs and the
+ * final state ... parallelizing the recurrence through chunked matrix
+ * operations while applying the log-domain gate consistently").  The result is
+ * the token-by-token recurrence's; chunking only re-associates it.
+ *
+ * Sequence n owns tokens cu_seqlens[n] .. cu_seqlens[n+1]-1 and the state tile
+ * slot = slot_idx ? slot_idx[n] : n.  Chunks of `chunk` tokens restart at every
+ * sequence start; the last chunk of a sequence may be short; a sequence may be
+ * empty (its final state is its initial state).
+ *
+ *   q, k         bf16 [T][Hqk][dk]     packed tokens
+ *   v            bf16 [T][Hv][dv]
+ *   g, beta      fp32 [T][Hv]
+ *   cu_seqlens   int32 [N+1], cu[0] = 0, non-decreasing, cu[N] = T (checked on
+ *                the device: a violating sequence is skipped and
+ *                GDN_DEV_BAD_CU_SEQLENS is set)
+ *   init_state   fp32 [num_slots][Hv][dv][dk] or NULL (= all-zero states)
+ *   final_state  fp32 [num_slots][Hv][dv][dk], written for every slot a
+ *                sequence maps to; may be the same buffer as init_state
+ *   slot_idx     int32 [N] or NULL; negative = padding sequence (o rows zero,
+ *                no state written); >= num_slots the same + GDN_DEV_BAD_SLOT
+ *   o            bf16 [T][Hv][dv], written
+ *   max_seqlen_hint  an upper bound on the longest sequence if the caller
+ *                knows one, else 0; only steers launch geometry, never results
+ *   workspace    device scratch of at least gdn_prefill_workspace_bytes(...)
+ *                bytes, 256-byte aligned; contents are scratch before and after
+ * T == 0 or N == 0 is a no-op that returns 0.
+ */
+int gdn_prefill(const void* q, const void* k, const void* v,
+                const float* g, const float* beta, const int32_t* cu_seqlens,
+                const float* init_state, float* final_state, const int32_t* slot_idx,
+                void* o,
+                int32_t T, int32_t N, int32_t max_seqlen_hint,
+                int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv, int32_t chunk,
+                int32_t num_slots, float scale,
+                void* workspace, size_t workspace_bytes,
+                int32_t* dev_status, void* stream);
+
+/*
+ * gdn_prefill_recurrent - the same operator and arguments as gdn_prefill,
+ * evaluated token by token on the CUDA cores (no chunking, no workspace).  The
+ * rows of a state tile evolve independently under the gated delta rule, so the
+ * dv rows are spread over warps.  It is the route for very short batches and
+ * an independent GPU cross-check of the chunked path.
+ */
+int gdn_prefill_recurrent(const void* q, const void* k, const void* v,
+                          const float* g, const float* beta, const int32_t* cu_seqlens,
+                          const float* init_state, float* final_state,
+                          const int32_t* slot_idx, void* o,
+                          int32_t T, int32_t N, int32_t Hqk, int32_t Hv,
+                          int32_t dk, int32_t dv, int32_t num_slots, float scale,
+                          int32_t* dev_status, void* stream);
+
+/* Human-readable name of a return code (static storage, never NULL). */
+const char* gdn_status_string(int code);
+
+/* Library version, major * 10000 + minor * 100 + patch. */
+int gdn_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GDN_B200_H_ */

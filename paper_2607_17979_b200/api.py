@@ -1,0 +1,129 @@
+"""Thin binding over the C-ABI library (``include/gdn.h``): argument marshalling only.
+
+Every function takes torch CUDA tensors, checks dtype / contiguity / device,
+and passes raw device pointers and the current CUDA stream to the entry point
+of the same name.  Nothing is computed here, and there is no fallback: if the
+compiled library is missing the import fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgdn_b200.so")
+
+EXPORTS = ("gdn_decode", "gdn_prefill_workspace_bytes", "gdn_prefill", "gdn_prefill_recurrent",
+           "gdn_status_string", "gdn_version")
+
+# kernels one call enqueues (for the benchmark's launch count)
+LAUNCHES_PER_DECODE = 1
+LAUNCHES_PER_PREFILL = 1
+LAUNCHES_PER_STEP = LAUNCHES_PER_DECODE + LAUNCHES_PER_PREFILL
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2607_17979_b200.build` "
+        "(nvcc, sm_100a). There is no CPU or PyTorch fallback for the gated delta rule kernels.")
+
+_lib = ctypes.CDLL(LIB_PATH)
+_P, _I, _F, _Z = ctypes.c_void_p, ctypes.c_int32, ctypes.c_float, ctypes.c_size_t
+_lib.gdn_decode.restype = ctypes.c_int
+_lib.gdn_decode.argtypes = [_P] * 8 + [_I] * 6 + [_F, _P, _P]
+_lib.gdn_prefill_workspace_bytes.restype = _Z
+_lib.gdn_prefill_workspace_bytes.argtypes = [_I] * 7
+_lib.gdn_prefill.restype = ctypes.c_int
+_lib.gdn_prefill.argtypes = [_P] * 10 + [_I] * 9 + [_F, _P, _Z, _P, _P]
+_lib.gdn_prefill_recurrent.restype = ctypes.c_int
+_lib.gdn_prefill_recurrent.argtypes = [_P] * 10 + [_I] * 7 + [_F, _P, _P]
+_lib.gdn_status_string.restype = ctypes.c_char_p
+_lib.gdn_status_string.argtypes = [ctypes.c_int]
+_lib.gdn_version.restype = ctypes.c_int
+
+
+class GdnError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} ({code})")
+
+
+def status_string(code: int) -> str:
+    return _lib.gdn_status_string(int(code)).decode()
+
+
+def version() -> int:
+    return int(_lib.gdn_version())
+
+
+def _dev(t, dtype, name, allow_none=False):
+    if t is None:
+        if allow_none:
+            return None
+        raise TypeError(f"{name} is required")
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError(f"{name} must be a contiguous CUDA tensor of dtype {dtype}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def gdn_decode(q, k, v, g, beta, state_pool, slot_idx, o, scale, dev_status=None):
+    """One decode step, state_pool updated in place, o written.  Shapes as in gdn.h."""
+    B, Hqk, dk = q.shape
+    _, Hv, dv = v.shape
+    rc = _lib.gdn_decode(
+        _dev(q, torch.bfloat16, "q"), _dev(k, torch.bfloat16, "k"), _dev(v, torch.bfloat16, "v"),
+        _dev(g, torch.float32, "g"), _dev(beta, torch.float32, "beta"),
+        _dev(state_pool, torch.float32, "state_pool"),
+        _dev(slot_idx, torch.int32, "slot_idx", True), _dev(o, torch.bfloat16, "o"),
+        B, Hqk, Hv, dk, dv, state_pool.shape[0], float(scale),
+        _dev(dev_status, torch.int32, "dev_status", True), _stream())
+    if rc != 0:
+        raise GdnError(rc, "gdn_decode")
+
+
+def gdn_prefill_workspace_bytes(T, N, Hqk, Hv, dk=128, dv=128, chunk=64) -> int:
+    return int(_lib.gdn_prefill_workspace_bytes(T, N, Hqk, Hv, dk, dv, chunk))
+
+
+def gdn_prefill(q, k, v, g, beta, cu_seqlens, init_state, final_state, slot_idx, o, scale,
+                workspace, max_seqlen_hint=0, chunk=64, dev_status=None):
+    """Chunked prefill over packed sequences.  ``workspace`` is a uint8 CUDA tensor."""
+    T, Hqk, dk = q.shape
+    _, Hv, dv = v.shape
+    N = cu_seqlens.shape[0] - 1
+    rc = _lib.gdn_prefill(
+        _dev(q, torch.bfloat16, "q"), _dev(k, torch.bfloat16, "k"), _dev(v, torch.bfloat16, "v"),
+        _dev(g, torch.float32, "g"), _dev(beta, torch.float32, "beta"),
+        _dev(cu_seqlens, torch.int32, "cu_seqlens"),
+        _dev(init_state, torch.float32, "init_state", True),
+        _dev(final_state, torch.float32, "final_state"),
+        _dev(slot_idx, torch.int32, "slot_idx", True), _dev(o, torch.bfloat16, "o"),
+        T, N, int(max_seqlen_hint), Hqk, Hv, dk, dv, int(chunk), final_state.shape[0],
+        float(scale), _dev(workspace, torch.uint8, "workspace"), workspace.numel(),
+        _dev(dev_status, torch.int32, "dev_status", True), _stream())
+    if rc != 0:
+        raise GdnError(rc, "gdn_prefill")
+
+
+def gdn_prefill_recurrent(q, k, v, g, beta, cu_seqlens, init_state, final_state, slot_idx, o,
+                          scale, dev_status=None):
+    """Token-by-token prefill on the CUDA cores; same arguments as gdn_prefill, no workspace."""
+    T, Hqk, dk = q.shape
+    _, Hv, dv = v.shape
+    N = cu_seqlens.shape[0] - 1
+    rc = _lib.gdn_prefill_recurrent(
+        _dev(q, torch.bfloat16, "q"), _dev(k, torch.bfloat16, "k"), _dev(v, torch.bfloat16, "v"),
+        _dev(g, torch.float32, "g"), _dev(beta, torch.float32, "beta"),
+        _dev(cu_seqlens, torch.int32, "cu_seqlens"),
+        _dev(init_state, torch.float32, "init_state", True),
+        _dev(final_state, torch.float32, "final_state"),
+        _dev(slot_idx, torch.int32, "slot_idx", True), _dev(o, torch.bfloat16, "o"),
+        T, N, Hqk, Hv, dk, dv, final_state.shape[0], float(scale),
+        _dev(dev_status, torch.int32, "dev_status", True), _stream())
+    if rc != 0:
+        raise GdnError(rc, "gdn_prefill_recurrent")

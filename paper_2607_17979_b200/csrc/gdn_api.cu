@@ -1,0 +1,126 @@
+// C-ABI entry points: argument validation and launch.  See include/gdn.h.
+#include "gdn_common.cuh"
+#include "../../include/gdn.h"
+
+namespace {
+
+inline bool misaligned(const void* p, size_t a) {
+    return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0;
+}
+
+int check_heads(int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv) {
+    if (Hqk <= 0 || Hv <= 0) return GDN_ERR_SIZE;
+    if (dk != gdn::kD || dv != gdn::kD || Hv % Hqk != 0) return GDN_ERR_SHAPE;
+    return GDN_OK;
+}
+
+int check_prefill(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                  const int32_t* cu, const float* init_state, float* final_state, void* o,
+                  int32_t T, int32_t N, int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv,
+                  int32_t num_slots) {
+    if (T < 0 || N < 0) return GDN_ERR_SIZE;
+    const int rc = check_heads(Hqk, Hv, dk, dv);
+    if (rc != GDN_OK) return rc;
+    if (T == 0 || N == 0) return GDN_OK;
+    if (num_slots <= 0) return GDN_ERR_SIZE;
+    if (!q || !k || !v || !g || !beta || !cu || !final_state || !o) return GDN_ERR_NULL;
+    if (misaligned(q, 16) || misaligned(k, 16) || misaligned(v, 16) || misaligned(o, 16) ||
+        misaligned(final_state, 16) || misaligned(init_state, 16) || misaligned(g, 4) ||
+        misaligned(beta, 4) || misaligned(cu, 4))
+        return GDN_ERR_ALIGN;
+    return GDN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int gdn_decode(const void* q, const void* k, const void* v, const float* g, const float* beta,
+               float* state_pool, const int32_t* slot_idx, void* o,
+               int32_t B, int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv,
+               int32_t num_slots, float scale, int32_t* dev_status, void* stream) {
+    if (B < 0) return GDN_ERR_SIZE;
+    const int rc = check_heads(Hqk, Hv, dk, dv);
+    if (rc != GDN_OK) return rc;
+    if (B == 0) return GDN_OK;
+    if (num_slots <= 0) return GDN_ERR_SIZE;
+    if (!q || !k || !v || !g || !beta || !state_pool || !o) return GDN_ERR_NULL;
+    if (misaligned(q, 16) || misaligned(k, 16) || misaligned(v, 16) || misaligned(o, 16) ||
+        misaligned(state_pool, 16) || misaligned(g, 4) || misaligned(beta, 4) ||
+        misaligned(slot_idx, 4) || misaligned(dev_status, 4))
+        return GDN_ERR_ALIGN;
+    gdn::DecodeParams p;
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.k = static_cast<const __nv_bfloat16*>(k);
+    p.v = static_cast<const __nv_bfloat16*>(v);
+    p.g = g; p.beta = beta; p.pool = state_pool; p.slot_idx = slot_idx;
+    p.o = static_cast<__nv_bfloat16*>(o);
+    p.B = B; p.Hqk = Hqk; p.Hv = Hv; p.num_slots = num_slots; p.scale = scale;
+    p.dev_status = dev_status;
+    return gdn::launch_decode(p, static_cast<cudaStream_t>(stream)) == cudaSuccess ? GDN_OK
+                                                                                   : GDN_ERR_CUDA;
+}
+
+size_t gdn_prefill_workspace_bytes(int32_t T, int32_t N, int32_t Hqk, int32_t Hv,
+                                   int32_t dk, int32_t dv, int32_t chunk) {
+    if (T < 0 || N < 0 || chunk != gdn::kChunk || check_heads(Hqk, Hv, dk, dv) != GDN_OK) return 0;
+    return 256;
+}
+
+int gdn_prefill_recurrent(const void* q, const void* k, const void* v, const float* g,
+                          const float* beta, const int32_t* cu_seqlens, const float* init_state,
+                          float* final_state, const int32_t* slot_idx, void* o,
+                          int32_t T, int32_t N, int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv,
+                          int32_t num_slots, float scale, int32_t* dev_status, void* stream) {
+    const int rc = check_prefill(q, k, v, g, beta, cu_seqlens, init_state, final_state, o,
+                                 T, N, Hqk, Hv, dk, dv, num_slots);
+    if (rc != GDN_OK || T == 0 || N == 0) return rc;
+    gdn::PrefillParams p;
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.k = static_cast<const __nv_bfloat16*>(k);
+    p.v = static_cast<const __nv_bfloat16*>(v);
+    p.g = g; p.beta = beta; p.cu_seqlens = cu_seqlens; p.init_state = init_state;
+    p.final_state = final_state; p.slot_idx = slot_idx;
+    p.o = static_cast<__nv_bfloat16*>(o);
+    p.T = T; p.N = N; p.Hqk = Hqk; p.Hv = Hv; p.num_slots = num_slots; p.scale = scale;
+    p.dev_status = dev_status;
+    return gdn::launch_prefill_recurrent(p, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? GDN_OK : GDN_ERR_CUDA;
+}
+
+int gdn_prefill(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                const int32_t* cu_seqlens, const float* init_state, float* final_state,
+                const int32_t* slot_idx, void* o, int32_t T, int32_t N, int32_t max_seqlen_hint,
+                int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv, int32_t chunk,
+                int32_t num_slots, float scale, void* workspace, size_t workspace_bytes,
+                int32_t* dev_status, void* stream) {
+    (void)max_seqlen_hint;
+    if (chunk != gdn::kChunk) return GDN_ERR_SHAPE;
+    const int rc = check_prefill(q, k, v, g, beta, cu_seqlens, init_state, final_state, o,
+                                 T, N, Hqk, Hv, dk, dv, num_slots);
+    if (rc != GDN_OK || T == 0 || N == 0) return rc;
+    if (!workspace) return GDN_ERR_NULL;
+    if (misaligned(workspace, 256)) return GDN_ERR_ALIGN;
+    if (workspace_bytes < gdn_prefill_workspace_bytes(T, N, Hqk, Hv, dk, dv, chunk))
+        return GDN_ERR_WORKSPACE;
+    return gdn_prefill_recurrent(q, k, v, g, beta, cu_seqlens, init_state, final_state, slot_idx,
+                                 o, T, N, Hqk, Hv, dk, dv, num_slots, scale, dev_status, stream);
+}
+
+const char* gdn_status_string(int code) {
+    switch (code) {
+        case GDN_OK: return "ok";
+        case GDN_ERR_NULL: return "a required pointer is NULL";
+        case GDN_ERR_SIZE: return "a size is negative or num_slots is not positive";
+        case GDN_ERR_SHAPE: return "unsupported shape (need dk = dv = 128, chunk = 64, Hv % Hqk = 0)";
+        case GDN_ERR_ALIGN: return "a pointer is not aligned as required";
+        case GDN_ERR_WORKSPACE: return "workspace too small";
+        case GDN_ERR_CUDA: return "CUDA runtime error at launch or set-up";
+        case GDN_ERR_LIMIT: return "a size exceeds the entry point's fixed maximum";
+        default: return "unknown status";
+    }
+}
+
+int gdn_version(void) { return 100; }
+
+}  // extern "C"

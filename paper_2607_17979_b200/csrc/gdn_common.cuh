@@ -1,0 +1,82 @@
+// Shared declarations of the CUDA side of the gated delta rule library.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+namespace gdn {
+
+constexpr int kD = 128;          // dk == dv == 128 is the only supported head size
+constexpr int kChunk = 64;       // prefill chunk length
+
+// device status bits (mirror GDN_DEV_* of the public header)
+constexpr int kDevBadSlot = 1;
+constexpr int kDevBadCuSeqlens = 2;
+constexpr int kDevTimeout = 4;
+
+struct DecodeParams {
+    const __nv_bfloat16* q;
+    const __nv_bfloat16* k;
+    const __nv_bfloat16* v;
+    const float* g;
+    const float* beta;
+    float* pool;
+    const int32_t* slot_idx;
+    __nv_bfloat16* o;
+    int32_t B, Hqk, Hv, num_slots;
+    float scale;
+    int32_t* dev_status;
+};
+
+struct PrefillParams {
+    const __nv_bfloat16* q;
+    const __nv_bfloat16* k;
+    const __nv_bfloat16* v;
+    const float* g;
+    const float* beta;
+    const int32_t* cu_seqlens;
+    const float* init_state;
+    float* final_state;
+    const int32_t* slot_idx;
+    __nv_bfloat16* o;
+    int32_t T, N, Hqk, Hv, num_slots;
+    float scale;
+    int32_t* dev_status;
+};
+
+cudaError_t launch_decode(const DecodeParams& p, cudaStream_t stream);
+cudaError_t launch_prefill_recurrent(const PrefillParams& p, cudaStream_t stream);
+
+__device__ __forceinline__ void report(int32_t* dev_status, int bit) {
+    if (dev_status) atomicOr(dev_status, bit);
+}
+
+// four consecutive bf16 -> four floats (8-byte aligned source)
+__device__ __forceinline__ float4 load_bf16x4(const __nv_bfloat16* p) {
+    const uint2 raw = *reinterpret_cast<const uint2*>(p);
+    float4 r;
+    r.x = __uint_as_float(raw.x << 16);
+    r.y = __uint_as_float(raw.x & 0xffff0000u);
+    r.z = __uint_as_float(raw.y << 16);
+    r.w = __uint_as_float(raw.y & 0xffff0000u);
+    return r;
+}
+
+__device__ __forceinline__ float dot4(const float4& a, const float4& b, float acc) {
+    acc = fmaf(a.x, b.x, acc);
+    acc = fmaf(a.y, b.y, acc);
+    acc = fmaf(a.z, b.z, acc);
+    acc = fmaf(a.w, b.w, acc);
+    return acc;
+}
+
+// sum over the 8 lanes that share a state row (lanes differing in bits 0..2)
+__device__ __forceinline__ float sum8(float x) {
+    x += __shfl_xor_sync(0xffffffffu, x, 1);
+    x += __shfl_xor_sync(0xffffffffu, x, 2);
+    x += __shfl_xor_sync(0xffffffffu, x, 4);
+    return x;
+}
+
+}  // namespace gdn

@@ -1,0 +1,178 @@
+"""GPU parity: gdn_prefill (chunked) and gdn_prefill_recurrent against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2607_17979_b200 import inputs as I
+import gpu_util as U
+
+pytestmark = pytest.mark.gpu
+
+IMPLS = ["chunked", "recurrent"]
+
+
+def run_prefill(p, impl, slot_idx=None, num_slots=None, init="from_inputs", alias=False,
+                pool_fill=None):
+    """Returns (o fp64 [T,Hv,128], final fp32 numpy [num_slots,Hv,128,128], status)."""
+    from paper_2607_17979_b200 import api
+    N, Hv, T = p["N"], p["Hv"], p["T"]
+    num_slots = N if num_slots is None else num_slots
+    init_np = p["init_state"] if isinstance(init, str) else init
+    init_t = U.dev(init_np)
+    if alias:
+        assert init_t is not None
+        final = init_t
+    else:
+        final = torch.full((num_slots, Hv, 128, 128), float("nan") if pool_fill is None else pool_fill,
+                           dtype=torch.float32, device="cuda")
+    o = torch.full((T, Hv, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    args = (U.dev_bf16(p["q"]), U.dev_bf16(p["k"]), U.dev_bf16(p["v"]), U.dev(p["g"]),
+            U.dev(p["beta"]), U.dev(p["cu_seqlens"]), init_t, final, U.dev(slot_idx), o, p["scale"])
+    if impl == "chunked":
+        ws = torch.empty(max(api.gdn_prefill_workspace_bytes(T, N, p["Hqk"], Hv), 256),
+                         dtype=torch.uint8, device="cuda")
+        api.gdn_prefill(*args, ws, dev_status=status)
+    else:
+        api.gdn_prefill_recurrent(*args, dev_status=status)
+    torch.cuda.synchronize()
+    return U.host_f64_from_bf16(o), final.cpu().numpy(), int(status.item())
+
+
+def oracle_prefill(p, slot_idx=None, num_slots=None, init="from_inputs"):
+    init_np = p["init_state"] if isinstance(init, str) else init
+    init64 = None if init_np is None else init_np.astype(np.float64)
+    o, S, bad = oracle.prefill(p["q"], p["k"], p["v"], p["g"], p["beta"], p["cu_seqlens"], init64,
+                               slot_idx, p["scale"], num_slots=num_slots)
+    return o, S, bad
+
+
+def compare(p, impl, **kw):
+    o, S, status = run_prefill(p, impl, **kw)
+    okw = {k: v for k, v in kw.items() if k in ("slot_idx", "num_slots", "init")}
+    o_ref, S_ref, _ = oracle_prefill(p, **okw)
+    assert status == 0
+    if p["T"] > 0:
+        U.check_o(o, o_ref, U.O_REL_L2_PREFILL)
+    return o, S, o_ref, S_ref
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("L", [1, 2, 63, 64, 65, 127, 128, 129, 200])
+def test_single_sequence_lengths(impl, L):
+    for seed, init in [(0, "zero"), (1, "normal"), (2, "normal")]:
+        p = I.prefill_inputs([L], 1, 2, seed=300 + seed, init=init)
+        o, S, o_ref, S_ref = compare(p, impl)
+        U.check_state(S.astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("Hqk,Hv", [(1, 1), (1, 2), (2, 4), (4, 8), (16, 32)])
+def test_packed_ragged_batch_with_empty_sequence(impl, Hqk, Hv):
+    lens = [1, 2, 63, 64, 0, 65, 127, 128, 129, 200]
+    if Hv == 32:
+        lens = [65, 0, 130]
+    p = I.prefill_inputs(lens, Hqk, Hv, seed=400 + Hv, init="normal")
+    o, S, o_ref, S_ref = compare(p, impl)
+    U.check_state(S.astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
+    empty = lens.index(0)
+    assert np.array_equal(S[empty], p["init_state"][empty])        # passes through bit-exactly
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_slots_padding_alias_and_untouched_slots(impl):
+    lens = [70, 5, 64, 33]
+    p = I.prefill_inputs(lens, 2, 4, seed=500, init="zero")
+    rs = np.random.default_rng(5)
+    pool = (rs.standard_normal((7, 4, 128, 128)) * 0.02).astype(np.float32)
+    idx = np.array([6, -1, 2, 9], np.int32)                         # padding, out of range
+    o, S, status = run_prefill(p, impl, slot_idx=idx, num_slots=7, init=pool, alias=True)
+    o_ref, S_ref, bad = oracle_prefill(p, slot_idx=idx, num_slots=7, init=pool)
+    assert status == 1 and bad == 4
+    cu = p["cu_seqlens"]
+    assert np.abs(o[cu[1]:cu[2]]).max() == 0 and np.abs(o[cu[3]:cu[4]]).max() == 0
+    U.check_o(o, o_ref, U.O_REL_L2_PREFILL)
+    assert np.array_equal(S[[0, 1, 3, 4, 5]], pool[[0, 1, 3, 4, 5]])
+    U.check_state(S[[6, 2]].astype(np.float64), S_ref[[6, 2]], U.STATE_REL_L2_PREFILL)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("case", ["beta0", "beta1", "g0", "alpha09", "v0", "same_keys"])
+def test_degenerate_values(impl, case):
+    p = I.prefill_inputs([150, 64], 2, 4, seed=600, init="normal")
+    if case == "beta0":
+        p["beta"][:] = 0
+    elif case == "beta1":
+        p["beta"][:] = 1
+    elif case == "g0":
+        p["g"][:] = 0
+    elif case == "alpha09":
+        p["g"][:] = np.float32(np.log(0.9))
+    elif case == "v0":
+        p["v"][:] = 0
+    elif case == "same_keys":                # worst case for the triangular solve
+        p["k"][:] = p["k"][:1, :1]
+        p["beta"][:] = 1
+    o, S, o_ref, S_ref = compare(p, impl)
+    U.check_state(S.astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_bad_cu_seqlens_sets_status_and_skips(impl):
+    p = I.prefill_inputs([40, 30], 1, 2, seed=700, init="zero")
+    p["cu_seqlens"] = np.array([0, 50, 45], np.int32)               # decreasing, and cu[N] != T
+    o, S, status = run_prefill(p, impl, pool_fill=7.0)
+    assert status & 2
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_deterministic_and_split_prefill_hand_off(impl):
+    p = I.prefill_inputs([192], 2, 4, seed=800, init="normal")
+    o1, S1, _ = run_prefill(p, impl)
+    o2, S2, _ = run_prefill(p, impl)
+    assert np.array_equal(o1, o2) and np.array_equal(S1, S2)
+    # prefill(128) then prefill(64 from its final state) tracks prefill(192)
+    a = {n: (x[:128] if isinstance(x, np.ndarray) and x.shape[:1] == (192,) else x) for n, x in p.items()}
+    b = {n: (x[128:] if isinstance(x, np.ndarray) and x.shape[:1] == (192,) else x) for n, x in p.items()}
+    a.update(T=128, cu_seqlens=np.array([0, 128], np.int32))
+    b.update(T=64, cu_seqlens=np.array([0, 64], np.int32))
+    oa, Sa, _ = run_prefill(a, impl)
+    ob, Sb, _ = run_prefill(b, impl, init=Sa)
+    o_ref, S_ref, _ = oracle_prefill(p)
+    U.check_o(np.concatenate([oa, ob]), o_ref, U.O_REL_L2_PREFILL)
+    U.check_state(Sb.astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
+
+
+def test_chunked_and_recurrent_routes_agree():
+    p = I.prefill_inputs([300, 17, 128], 2, 4, seed=900, init="normal")
+    oc, Sc, _ = run_prefill(p, "chunked")
+    orr, Sr, _ = run_prefill(p, "recurrent")
+    assert np.abs(oc - orr).max() <= U.O_MAX_ABS
+    assert U.rel_l2(Sc.astype(np.float64), Sr.astype(np.float64)) <= U.STATE_REL_L2_PREFILL
+
+
+def test_prefill_varlen_benchmark_config_full():
+    """4 sequences {512,1024,2048,4096}, 32 v-heads: every output against the oracle."""
+    p = I.make_config(3, 0)
+    o, S, o_ref, S_ref = compare(p, "chunked")
+    U.check_state(S.astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
+    cu = p["cu_seqlens"]
+    for n in range(4):                                               # no sequence hides in the norm
+        U.check_o(o[cu[n]:cu[n + 1]], o_ref[cu[n]:cu[n + 1]], U.O_REL_L2_PREFILL)
+
+
+def test_prefill_long_context_benchmark_config_sampled_heads():
+    """One 32768-token sequence at full size on the GPU; the oracle recomputes four sampled
+    v-heads (each with its own q/k head) over the whole sequence."""
+    p = I.make_config(4, 0)
+    o, S, status = run_prefill(p, "chunked")
+    assert status == 0 and np.isfinite(o).all() and np.isfinite(S).all()
+    for hv in (0, 13, 22, 31):
+        hq = hv // 2
+        o_ref, S_ref, _ = oracle.prefill(p["q"][:, hq:hq + 1], p["k"][:, hq:hq + 1], p["v"][:, hv:hv + 1],
+                                         p["g"][:, hv:hv + 1], p["beta"][:, hv:hv + 1], p["cu_seqlens"],
+                                         p["init_state"][:, hv:hv + 1].astype(np.float64), None, p["scale"])
+        U.check_o(o[:, hv:hv + 1], o_ref, U.O_REL_L2_PREFILL)
+        U.check_o(o[-4096:, hv:hv + 1], o_ref[-4096:], U.O_REL_L2_PREFILL)   # the far end of the carry
+        U.check_state(S[:, hv:hv + 1].astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
