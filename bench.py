@@ -83,7 +83,7 @@ class ClockSampler:
             os.close(fd)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                 "-i", str(self.gpu), "-lms", "50"], stdout=open(self.path, "w"),
+                 "-i", str(self.gpu), "-lms", "20"], stdout=open(self.path, "w"),
                 stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -284,12 +284,14 @@ def run_ours(args):
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t[0]), float(t[1])
 
+    # clocks are sampled from before the warm-up to after the timed steps (the GPU is under the
+    # same load throughout; the timed steps alone can be shorter than one sampling period)
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
     dec_ms, pre_ms = timed_region(step)
-    clocks = sampler.stop() if rank == 0 else None
     e2e_dec_ms, e2e_pre_ms = timed_region(e2e_step)
+    clocks = sampler.stop() if rank == 0 else None
     assert int(status.item()) == 0, "device status flagged during the benchmark"
 
     if rank == 0:
@@ -352,8 +354,8 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
     if args.impl == "reference":

@@ -20,7 +20,7 @@ EXPORTS = ("gdn_decode", "gdn_prefill_workspace_bytes", "gdn_prefill", "gdn_pref
 
 # kernels one call enqueues (for the benchmark's launch count)
 LAUNCHES_PER_DECODE = 1
-LAUNCHES_PER_PREFILL = 1
+LAUNCHES_PER_PREFILL = 3
 LAUNCHES_PER_STEP = LAUNCHES_PER_DECODE + LAUNCHES_PER_PREFILL
 
 if not os.path.exists(LIB_PATH):

@@ -1,5 +1,6 @@
 // C-ABI entry points: argument validation and launch.  See include/gdn.h.
 #include "gdn_common.cuh"
+#include "gdn_prefill_chunk.cuh"
 #include "../../include/gdn.h"
 
 namespace {
@@ -64,7 +65,7 @@ int gdn_decode(const void* q, const void* k, const void* v, const float* g, cons
 size_t gdn_prefill_workspace_bytes(int32_t T, int32_t N, int32_t Hqk, int32_t Hv,
                                    int32_t dk, int32_t dv, int32_t chunk) {
     if (T < 0 || N < 0 || chunk != gdn::kChunk || check_heads(Hqk, Hv, dk, dv) != GDN_OK) return 0;
-    return 256;
+    return gdn::workspace_layout(T, N, Hv).total;
 }
 
 int gdn_prefill_recurrent(const void* q, const void* k, const void* v, const float* g,
@@ -103,8 +104,20 @@ int gdn_prefill(const void* q, const void* k, const void* v, const float* g, con
     if (misaligned(workspace, 256)) return GDN_ERR_ALIGN;
     if (workspace_bytes < gdn_prefill_workspace_bytes(T, N, Hqk, Hv, dk, dv, chunk))
         return GDN_ERR_WORKSPACE;
-    return gdn_prefill_recurrent(q, k, v, g, beta, cu_seqlens, init_state, final_state, slot_idx,
-                                 o, T, N, Hqk, Hv, dk, dv, num_slots, scale, dev_status, stream);
+    gdn::ChunkedParams cp;
+    gdn::PrefillParams& p = cp.p;
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.k = static_cast<const __nv_bfloat16*>(k);
+    p.v = static_cast<const __nv_bfloat16*>(v);
+    p.g = g; p.beta = beta; p.cu_seqlens = cu_seqlens; p.init_state = init_state;
+    p.final_state = final_state; p.slot_idx = slot_idx;
+    p.o = static_cast<__nv_bfloat16*>(o);
+    p.T = T; p.N = N; p.Hqk = Hqk; p.Hv = Hv; p.num_slots = num_slots; p.scale = scale;
+    p.dev_status = dev_status;
+    cp.ws = static_cast<uint8_t*>(workspace);
+    cp.lay = gdn::workspace_layout(T, N, Hv);
+    return gdn::launch_prefill_chunked(cp, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? GDN_OK : GDN_ERR_CUDA;
 }
 
 const char* gdn_status_string(int code) {

@@ -1,0 +1,76 @@
+// Chunked prefill: shared layout of the workspace and of the per-(chunk, v-head) record.
+//
+// Inside a chunk of C = 64 tokens entering with state S0 (dv x dk), with
+// b_r = sum_{i<=r} g_i (inclusive, chunk-local) the gated delta rule unrolls to
+//
+//   A_ri = beta_r e^{b_r-b_i} (k_r.k_i)  (i <  r),   T = (I + A)^{-1}
+//   P_ri =        e^{b_r-b_i} (q_r.k_i)  (i <= r)
+//   W  = T diag(beta e^b) K   (C x dk),   U~ = T diag(beta) V   (C x dv)
+//   U  = U~ - W S0^T
+//   O  = scale ( diag(e^b) Q S0^T + P U )
+//   S' = e^{b_C} S0 + U^T diag(e^{b_C-b}) K
+//
+// Three launches: a prep kernel builds the chunk table from cu_seqlens; the
+// intra-chunk kernel (one CTA per chunk and v-head, all chunks in parallel)
+// computes W, U~, P and b with tcgen05 GEMMs and an fp32 triangular solve and
+// writes them as a record; the state-pass kernel (one CTA per sequence and
+// v-head) walks the chunks in order carrying S in fp32 registers.
+#pragma once
+#include "gdn_common.cuh"
+#include <cuda.h>
+
+namespace gdn {
+
+// One record per (chunk, v-head), written by the intra-chunk kernel in exactly the
+// byte image the state-pass kernel wants in shared memory (one linear bulk copy):
+//   [0, 16384)      W  as two K-major 128B-swizzled halves [64 tokens][64 dk] bf16
+//   [16384, 24576)  P  as one K-major 128B-swizzled tile   [64 r][64 i]      bf16
+//   [24576, 57344)  U~ as [16 token-groups][128 dv][4 tokens] fp32
+//   [57344, 57600)  b  as [64] fp32 (rows past the chunk's length repeat the last value)
+constexpr uint32_t kRecW = 0;
+constexpr uint32_t kRecP = 16384;
+constexpr uint32_t kRecU = 24576;
+constexpr uint32_t kRecB = 57344;
+constexpr uint32_t kRecBytes = 57600;
+
+struct ChunkInfo {      // 16 bytes
+    int32_t seq;        // sequence the chunk belongs to
+    int32_t t0;         // first packed token of the chunk
+    int32_t len;        // valid tokens (1..64)
+    int32_t pad;
+};
+
+// Workspace layout (all offsets multiples of 256 bytes):
+//   [0,256)                      int32 total_chunks
+//   seq_first[N+1]               int32: first chunk of each sequence (prefix sum); an invalid
+//                                sequence has zero chunks and seq_bad[n] = 1
+//   seq_bad[N]                   int32
+//   chunks[max_chunks]           ChunkInfo
+//   records[max_chunks][Hv]      kRecBytes each
+struct WorkspaceLayout {
+    size_t seq_first, seq_bad, chunks, records, total;
+    int32_t max_chunks;
+};
+
+inline size_t round256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
+
+inline WorkspaceLayout workspace_layout(int32_t T, int32_t N, int32_t Hv) {
+    WorkspaceLayout w;
+    w.max_chunks = T / kChunk + N;
+    w.seq_first = 256;
+    w.seq_bad = w.seq_first + round256(sizeof(int32_t) * (static_cast<size_t>(N) + 1));
+    w.chunks = w.seq_bad + round256(sizeof(int32_t) * static_cast<size_t>(N ? N : 1));
+    w.records = w.chunks + round256(sizeof(ChunkInfo) * static_cast<size_t>(w.max_chunks ? w.max_chunks : 1));
+    w.total = w.records + static_cast<size_t>(w.max_chunks) * Hv * kRecBytes;
+    return w;
+}
+
+struct ChunkedParams {
+    PrefillParams p;
+    uint8_t* ws;
+    WorkspaceLayout lay;
+};
+
+cudaError_t launch_prefill_chunked(const ChunkedParams& cp, cudaStream_t stream);
+
+}  // namespace gdn
