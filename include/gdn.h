@@ -145,6 +145,41 @@ int gdn_prefill_recurrent(const void* q, const void* k, const void* v,
                           int32_t dk, int32_t dv, int32_t num_slots, float scale,
                           int32_t* dev_status, void* stream);
 
+/*
+ * gdn_prefill_static - gdn_prefill for callers that cannot allocate device
+ * memory.  (No counterpart in the paper: this is a deployment convenience of
+ * this library.)  Some callers are not allowed to call cudaMalloc: code running
+ * inside another framework's memory plan, a plugin that receives tensors but no
+ * allocator, a serving loop whose HBM is already fully assigned.  For them the
+ * scratch workspace comes from a fixed array inside the library's own device
+ * image, GDN_STATIC_WORKSPACE_BYTES large, which every GPU that loads the
+ * library holds until the process exits.
+ *
+ * Arguments and results are exactly gdn_prefill's, minus workspace and
+ * workspace_bytes; inputs and outputs are still the caller's buffers.
+ *   - A batch needing more scratch than the array holds
+ *     (gdn_prefill_workspace_bytes(...) > GDN_STATIC_WORKSPACE_BYTES) returns
+ *     GDN_ERR_LIMIT and nothing is launched.  With Hv = 32 the array covers up to
+ *     18 chunks of 64 tokens (floor(T/64) + N <= 18), e.g. 1024 tokens in 2 sequences.
+ *   - The call itself allocates and frees nothing.  The first call on each
+ *     device looks up the array's device address (one cudaGetSymbolAddress, with
+ *     that device current) and caches it; make that first call outside of any
+ *     stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous
+ *     call's contents; nothing in it needs to be zero on entry.  Calls that
+ *     overlap on the GPU (two streams, two threads) race on it: serialise them.
+ */
+#define GDN_STATIC_WORKSPACE_BYTES (32u << 20)
+size_t gdn_prefill_static_workspace_bytes(void);
+int gdn_prefill_static(const void* q, const void* k, const void* v,
+                       const float* g, const float* beta, const int32_t* cu_seqlens,
+                       const float* init_state, float* final_state, const int32_t* slot_idx,
+                       void* o,
+                       int32_t T, int32_t N, int32_t max_seqlen_hint,
+                       int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv, int32_t chunk,
+                       int32_t num_slots, float scale,
+                       int32_t* dev_status, void* stream);
+
 /* Human-readable name of a return code (static storage, never NULL). */
 const char* gdn_status_string(int code);
 

@@ -16,7 +16,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libgdn_b200.so")
 
 EXPORTS = ("gdn_decode", "gdn_prefill_workspace_bytes", "gdn_prefill", "gdn_prefill_recurrent",
-           "gdn_status_string", "gdn_version")
+           "gdn_prefill_static", "gdn_prefill_static_workspace_bytes", "gdn_status_string",
+           "gdn_version")
 
 # kernels one call enqueues (for the benchmark's launch count)
 LAUNCHES_PER_DECODE = 1
@@ -38,6 +39,10 @@ _lib.gdn_prefill.restype = ctypes.c_int
 _lib.gdn_prefill.argtypes = [_P] * 10 + [_I] * 9 + [_F, _P, _Z, _P, _P]
 _lib.gdn_prefill_recurrent.restype = ctypes.c_int
 _lib.gdn_prefill_recurrent.argtypes = [_P] * 10 + [_I] * 7 + [_F, _P, _P]
+_lib.gdn_prefill_static.restype = ctypes.c_int
+_lib.gdn_prefill_static.argtypes = [_P] * 10 + [_I] * 9 + [_F, _P, _P]
+_lib.gdn_prefill_static_workspace_bytes.restype = _Z
+_lib.gdn_prefill_static_workspace_bytes.argtypes = []
 _lib.gdn_status_string.restype = ctypes.c_char_p
 _lib.gdn_status_string.argtypes = [ctypes.c_int]
 _lib.gdn_version.restype = ctypes.c_int
@@ -127,3 +132,29 @@ def gdn_prefill_recurrent(q, k, v, g, beta, cu_seqlens, init_state, final_state,
         _dev(dev_status, torch.int32, "dev_status", True), _stream())
     if rc != 0:
         raise GdnError(rc, "gdn_prefill_recurrent")
+
+
+def gdn_prefill_static_workspace_bytes() -> int:
+    """Size of the scratch array built into the library (the limit gdn_prefill_static enforces)."""
+    return int(_lib.gdn_prefill_static_workspace_bytes())
+
+
+def gdn_prefill_static(q, k, v, g, beta, cu_seqlens, init_state, final_state, slot_idx, o, scale,
+                       max_seqlen_hint=0, chunk=64, dev_status=None):
+    """gdn_prefill without a caller-supplied workspace, for callers that may not allocate device
+    memory: the scratch is a fixed array inside the library.  Raises GdnError(-7) when the batch
+    needs more scratch than that array holds.  Calls sharing a device must not overlap."""
+    T, Hqk, dk = q.shape
+    _, Hv, dv = v.shape
+    N = cu_seqlens.shape[0] - 1
+    rc = _lib.gdn_prefill_static(
+        _dev(q, torch.bfloat16, "q"), _dev(k, torch.bfloat16, "k"), _dev(v, torch.bfloat16, "v"),
+        _dev(g, torch.float32, "g"), _dev(beta, torch.float32, "beta"),
+        _dev(cu_seqlens, torch.int32, "cu_seqlens"),
+        _dev(init_state, torch.float32, "init_state", True),
+        _dev(final_state, torch.float32, "final_state"),
+        _dev(slot_idx, torch.int32, "slot_idx", True), _dev(o, torch.bfloat16, "o"),
+        T, N, int(max_seqlen_hint), Hqk, Hv, dk, dv, int(chunk), final_state.shape[0],
+        float(scale), _dev(dev_status, torch.int32, "dev_status", True), _stream())
+    if rc != 0:
+        raise GdnError(rc, "gdn_prefill_static")
