@@ -3,6 +3,22 @@
 #include "gdn_prefill_chunk.cuh"
 #include "gdn_sm100.cuh"
 
+// Optional phase timing for development builds (-DGDN_PHASE_TIMING): thread 0 of one chosen CTA
+// accumulates clock64() deltas per phase and leaves them in the workspace header.
+#ifdef GDN_PHASE_TIMING
+#define PT_DECL long long pt_last = clock64(); long long pt_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+#define PT(k) do { if (threadIdx.x == 0) { const long long t_ = clock64(); pt_acc[k] += t_ - pt_last; pt_last = t_; } } while (0)
+#define PTI(k) do { const long long t_ = clock64(); pt_acc[k] += t_ - pt_last; pt_last = t_; } while (0)
+#define PTI_FLUSH(cond, off, n) do { if (cond) for (int i_ = 0; i_ < (n); ++i_) reinterpret_cast<long long*>(ws + (off))[i_] = pt_acc[i_]; } while (0)
+#define PT_FLUSH(cond, off, n) do { if (threadIdx.x == 0 && (cond)) for (int i_ = 0; i_ < (n); ++i_) reinterpret_cast<long long*>(ws + (off))[i_] = pt_acc[i_]; } while (0)
+#else
+#define PT_DECL
+#define PT(k)
+#define PTI(k)
+#define PTI_FLUSH(cond, off, n)
+#define PT_FLUSH(cond, off, n)
+#endif
+
 namespace gdn {
 using namespace sm100;
 
@@ -71,26 +87,149 @@ prefill_prep_kernel(const int32_t* __restrict__ cu, int32_t T, int32_t N, uint8_
 }
 
 // =============================================================================================
-// K1: intra-chunk quantities, one CTA (128 threads) per (chunk, v-head).
+// K1: intra-chunk quantities, one CTA (256 threads) per (chunk, v-head).
 // =============================================================================================
-constexpr int kIntraThreads = 128;
+constexpr int kIntraThreads = 256;
 constexpr uint32_t kIntraTmemCols = 256;
+constexpr int kLdA = 68;               // row stride (floats) of the fp32 A / T matrix
 // shared memory map (bytes from a 1024-aligned base)
 constexpr uint32_t kI_QK = 0;          // 2 halves x [128 rows x 128 B]: rows 0-63 Q, 64-127 K
 constexpr uint32_t kI_V = 32768;       // 2 halves x [64 x 128 B]
-constexpr uint32_t kI_Tw = 49152;      // [64 r x 64 i] bf16, K-major SW128
-constexpr uint32_t kI_Tu = 57344;      // T_u rounded to bf16 ...
-constexpr uint32_t kI_TuLo = 65536;    // ... and the bf16 remainder (T_u = hi + lo to ~2^-17)
+constexpr uint32_t kI_Tw = 49152;      // T diag(beta e^b)  [64 r x 64 i] bf16, K-major SW128
+constexpr uint32_t kI_Tu = 57344;      // T diag(beta) rounded to bf16 ...
+constexpr uint32_t kI_TuLo = 65536;    // ... and the bf16 remainder (hi + lo carries ~16 bits)
 constexpr uint32_t kI_P = 73728;       // P image staging
-constexpr uint32_t kI_AT = 81920;      // A transposed, fp32 [64 i][64 r]
-constexpr uint32_t kI_End = 81920 + 16384;
-constexpr uint32_t kIntraSmem = kI_End + 1024;   // + alignment slack
+constexpr uint32_t kI_A = 81920;       // A, then T in place: fp32 [64][kLdA]
+constexpr uint32_t kI_Scr = kI_A + 64 * kLdA * 4;      // solve scratch, fp32 [32][36]
+constexpr uint32_t kI_End = kI_Scr + 32 * 36 * 4;
+constexpr uint32_t kIntraSmem = kI_End + 1024;         // + alignment slack
 
 struct TensorMaps {
     CUtensorMap q, k, v;
 };
 
-__global__ void __launch_bounds__(kIntraThreads)
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// T = (I + A)^{-1} for the strictly lower-triangular 64x64 A in sA (row-major, stride kLdA),
+// in place, by 256 threads: four 16x16 diagonal blocks by forward substitution, then the
+// off-diagonal blocks by block elimination at block sizes 16 and 32
+//     [[Ta, 0], [X, Tb]],  X = -Tb (A_ba Ta).
+// fp32 throughout.  Ends with a __syncthreads().
+#ifdef GDN_PHASE_TIMING
+#define ST(k) do { if (tid == 0 && st_out) st_out[k] = clock64(); } while (0)
+#else
+#define ST(k)
+#endif
+__device__ __forceinline__ void solve_unit_lower_64(float* sA, float* scr, int tid, long long* st_out) {
+    ST(0);
+    // ---- diagonal blocks: thread (I, j) computes column j of (I + A_II)^{-1}, right-looking
+    if (tid < 64) {
+        const int I = tid >> 4, j = tid & 15;
+        float* blk = sA + (16 * I) * kLdA + 16 * I;
+        float t[16];
+#pragma unroll
+        for (int r = 0; r < 16; ++r) t[r] = (r == j) ? 1.f : 0.f;
+#pragma unroll
+        for (int i = 0; i < 15; ++i) {
+            const float ti = t[i];
+#pragma unroll
+            for (int r = i + 1; r < 16; ++r) t[r] = fmaf(-blk[r * kLdA + i], ti, t[r]);
+        }
+        __syncwarp();                      // every column of the block has read A_II
+#pragma unroll
+        for (int r = 0; r < 16; ++r) blk[r * kLdA + j] = t[r];
+    }
+    ST(1);
+    __syncthreads();
+    ST(2);
+    // ---- 16-blocks (1,0) and (3,2): two chains of two 16x16x16 products, 128 threads each,
+    //      thread = (row ty, two columns 2tx, 2tx+1)
+    {
+        const int pr = tid >> 7, t = tid & 127, ty = t >> 3, tx = t & 7;
+        const int I = 2 * pr + 1, J = 2 * pr;
+        float* X = scr + pr * (16 * 20);
+        float2 acc = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int k0 = 0; k0 < 16; k0 += 4) {
+            const float4 a = *reinterpret_cast<const float4*>(sA + (16 * I + ty) * kLdA + 16 * J + k0);
+            const float av[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                const float2 b = *reinterpret_cast<const float2*>(sA + (16 * J + k0 + kk) * kLdA + 16 * J + 2 * tx);
+                acc.x = fmaf(av[kk], b.x, acc.x); acc.y = fmaf(av[kk], b.y, acc.y);
+            }
+        }
+        *reinterpret_cast<float2*>(X + ty * 20 + 2 * tx) = acc;
+        __syncthreads();
+        ST(3);
+        acc = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int k0 = 0; k0 < 16; k0 += 4) {
+            const float4 a = *reinterpret_cast<const float4*>(sA + (16 * I + ty) * kLdA + 16 * I + k0);
+            const float av[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                const float2 b = *reinterpret_cast<const float2*>(X + (k0 + kk) * 20 + 2 * tx);
+                acc.x = fmaf(-av[kk], b.x, acc.x); acc.y = fmaf(-av[kk], b.y, acc.y);
+            }
+        }
+        *reinterpret_cast<float2*>(sA + (16 * I + ty) * kLdA + 16 * J + 2 * tx) = acc;
+    }
+    __syncthreads();
+    ST(4);
+    // ---- 32-block (1,0): Y = A_ba Ta, then X = -Tb Y; thread = (row ty, columns 4tx..4tx+3)
+    {
+        const int ty = tid >> 3, tx = tid & 7;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int k0 = 0; k0 < 32; k0 += 4) {
+            const float4 a = *reinterpret_cast<const float4*>(sA + (32 + ty) * kLdA + k0);
+            const float av[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                const float4 b = *reinterpret_cast<const float4*>(sA + (k0 + kk) * kLdA + 4 * tx);
+                acc.x = fmaf(av[kk], b.x, acc.x); acc.y = fmaf(av[kk], b.y, acc.y);
+                acc.z = fmaf(av[kk], b.z, acc.z); acc.w = fmaf(av[kk], b.w, acc.w);
+            }
+        }
+        *reinterpret_cast<float4*>(scr + ty * 36 + 4 * tx) = acc;
+        __syncthreads();
+        ST(5);
+        acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int k0 = 0; k0 < 32; k0 += 4) {
+            const float4 a = *reinterpret_cast<const float4*>(sA + (32 + ty) * kLdA + 32 + k0);
+            const float av[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                const float4 b = *reinterpret_cast<const float4*>(scr + (k0 + kk) * 36 + 4 * tx);
+                acc.x = fmaf(-av[kk], b.x, acc.x); acc.y = fmaf(-av[kk], b.y, acc.y);
+                acc.z = fmaf(-av[kk], b.z, acc.z); acc.w = fmaf(-av[kk], b.w, acc.w);
+            }
+        }
+        *reinterpret_cast<float4*>(sA + (32 + ty) * kLdA + 4 * tx) = acc;
+    }
+    __syncthreads();
+    ST(6);
+}
+
+// Lane 0 polls the mbarrier (bounded), the other lanes block at the warp barrier instead of
+// competing for issue slots; returns the same verdict on every lane.
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity) {
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity) ? 1 : 0;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+
+__device__ __forceinline__ uint32_t scale_bf16x2(uint32_t packed, float f) {
+    return pack_bf16(__uint_as_float(packed << 16) * f, __uint_as_float(packed & 0xffff0000u) * f);
+}
+
+__global__ void __launch_bounds__(kIntraThreads, 2)
 prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParams p, uint8_t* ws,
                      const WorkspaceLayout lay) {
     const int c = blockIdx.x;
@@ -107,9 +246,14 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
     __shared__ uint64_t bar_tma, bar_mma;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_flag;
-    __shared__ float s_g[kChunk], s_b[kChunk], s_beta[kChunk];
+    __shared__ __align__(16) float s_b2[kChunk];     // b_r log2(e): inclusive log-decay prefix
+    __shared__ __align__(16) float s_beta[kChunk];   // beta_r (0 past the chunk's length)
+    __shared__ __align__(16) float s_bg[kChunk];     // beta_r e^{b_r}
+    __shared__ __align__(16) float s_eb[kChunk];     // e^{b_r}
 
     const int tid = threadIdx.x, warp = tid >> 5;
+    const int colhalf = warp >> 2;                   // which 32 of the 64 accumulator columns
+    PT_DECL
     if (tid == 0) {
         mbar_init(&bar_tma, 1);
         mbar_init(&bar_mma, 1);
@@ -120,16 +264,44 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
         tmem_alloc(&tmem_base_s, kIntraTmemCols);
         tmem_relinquish();
     }
-    if (tid < kChunk) {
-        const bool valid = tid < ci.len;
-        const size_t th = static_cast<size_t>(ci.t0 + (valid ? tid : 0)) * p.Hv + hv;
-        s_g[tid] = valid ? p.g[th] : 0.f;
-        s_beta[tid] = valid ? p.beta[th] : 0.f;
+    if (warp == 1) {
+        // inclusive prefix sum of the log gates over the chunk (two tokens per lane); rows past
+        // the chunk's length get g = 0, beta = 0 and so change nothing downstream
+        const int lane = tid & 31;
+        float g0 = 0.f, g1 = 0.f, be0 = 0.f, be1 = 0.f;
+        if (2 * lane < ci.len) {
+            const size_t th = static_cast<size_t>(ci.t0 + 2 * lane) * p.Hv + hv;
+            g0 = p.g[th]; be0 = p.beta[th];
+        }
+        if (2 * lane + 1 < ci.len) {
+            const size_t th = static_cast<size_t>(ci.t0 + 2 * lane + 1) * p.Hv + hv;
+            g1 = p.g[th]; be1 = p.beta[th];
+        }
+        float incl = g0 + g1;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const float y = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += y;
+        }
+        const float kLog2e = 1.4426950408889634f;
+        const float b1 = incl, b0 = incl - g1;
+        const float bC = __shfl_sync(0xffffffffu, incl, 31);
+        s_b2[2 * lane] = b0 * kLog2e; s_b2[2 * lane + 1] = b1 * kLog2e;
+        s_beta[2 * lane] = be0; s_beta[2 * lane + 1] = be1;
+        const float e0 = ex2_approx(b0 * kLog2e), e1 = ex2_approx(b1 * kLog2e);
+        s_eb[2 * lane] = e0; s_eb[2 * lane + 1] = e1;
+        s_bg[2 * lane] = be0 * e0; s_bg[2 * lane + 1] = be1 * e1;
+        // decay vector of the record: e^{b_C - b_c}, then e^{b_C}
+        float* dec = reinterpret_cast<float*>(rec + kRecDecay);
+        dec[2 * lane] = ex2_approx((bC - b0) * kLog2e);
+        dec[2 * lane + 1] = ex2_approx((bC - b1) * kLog2e);
+        if (lane == 0) dec[kChunk] = ex2_approx(bC * kLog2e);
     }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = tmem_base_s;
+    PT(0);
 
     if (tid == 0) {
         mbar_expect_tx(&bar_tma, 32768 + 16384);
@@ -140,12 +312,7 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
         tma_load_2d(smem + kI_V, &maps.v, hv * kD, ci.t0, &bar_tma);
         tma_load_2d(smem + kI_V + 8192, &maps.v, hv * kD + 64, ci.t0, &bar_tma);
     }
-    if (tid < kChunk) {            // inclusive prefix sum of the log gates, in token order
-        float acc = 0.f;
-        for (int i = 0; i <= tid; ++i) acc += s_g[i];
-        s_b[tid] = acc;
-    }
-    if (!mbar_wait(&bar_tma, 0)) abort_flag = 1;
+    if (warp == 0 && !warp_wait(&bar_tma, 0)) abort_flag = 1;      // one warp polls, the rest block
     __syncthreads();
     if (abort_flag) {
         if (tid == 0) report(p.dev_status, kDevTimeout);
@@ -153,6 +320,7 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
         return;
     }
     tc_fence_after_sync();
+    PT(1);
 
     const uint32_t tG = tmem, tW = tmem + 64, tU = tmem + 128;
     const uint32_t sQK = smem_u32(smem + kI_QK);
@@ -167,7 +335,7 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
         }
         mma_commit(&bar_mma);
     }
-    if (!mbar_wait(&bar_mma, 0)) abort_flag = 1;
+    if (warp == 0 && !warp_wait(&bar_mma, 0)) abort_flag = 1;      // one warp polls, the rest block
     __syncthreads();
     if (abort_flag) {
         if (tid == 0) report(p.dev_status, kDevTimeout);
@@ -175,82 +343,118 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
         return;
     }
     tc_fence_after_sync();
+    PT(2);
 
-    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
-    float* sAT = reinterpret_cast<float*>(smem + kI_AT);
+    const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    float* sA = reinterpret_cast<float*>(smem + kI_A);
     {
-        const int r = tid & 63;
-        const float br = s_b[r];
-        const float beta_r = s_beta[r];
+        // Accumulator row of this thread: TMEM lane 32 (warp % 4) + lane; lanes 0-63 hold q.k
+        // rows (-> P), lanes 64-127 hold k.k rows (-> A).  The thread covers 32 of the 64 columns.
+        const int row = (warp & 3) * 32 + (tid & 31);
+        const int r = row & 63;
+        const bool is_p = row < 64;
+        const int cbase = colhalf * 32;
+        const float br2 = s_b2[r];
+        const float rowscale = is_p ? 1.f : s_beta[r];
+        const int limit = is_p ? r : r - 1;              // keep columns i <= limit
+        uint32_t xa[16], xb[16];
+        tmem_ld16(tG + lane_base + cbase, xa);
+        tmem_ld16(tG + lane_base + cbase + 16, xb);
+        tmem_wait_ld();
+        float val[32];
 #pragma unroll
-        for (int c0 = 0; c0 < 64; c0 += 16) {
-            uint32_t x[16];
-            tmem_ld16(tG + lane_base + c0, x);
-            tmem_wait_ld();
-            if (tid < 64) {        // P row r -> bf16 image
-                float pv[16];
+        for (int q4 = 0; q4 < 8; ++q4) {
+            const float4 bb = *reinterpret_cast<const float4*>(s_b2 + cbase + 4 * q4);
+            const float bv[4] = {bb.x, bb.y, bb.z, bb.w};
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int i = c0 + j;
-                    pv[j] = (i <= r) ? __expf(br - s_b[i]) * __uint_as_float(x[j]) : 0.f;
-                }
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint4 w;
-                    w.x = pack_bf16(pv[8 * h + 0], pv[8 * h + 1]);
-                    w.y = pack_bf16(pv[8 * h + 2], pv[8 * h + 3]);
-                    w.z = pack_bf16(pv[8 * h + 4], pv[8 * h + 5]);
-                    w.w = pack_bf16(pv[8 * h + 6], pv[8 * h + 7]);
-                    *reinterpret_cast<uint4*>(smem + kI_P + sw128_offset(r, (c0 >> 3) + h)) = w;
-                }
-            } else {               // A row r, stored transposed for the solve
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int i = c0 + j;
-                    sAT[i * 64 + r] =
-                        (i < r) ? beta_r * __expf(br - s_b[i]) * __uint_as_float(x[j]) : 0.f;
-                }
+            for (int e = 0; e < 4; ++e) {
+                const int jj = 4 * q4 + e;
+                const float x = __uint_as_float(jj < 16 ? xa[jj] : xb[jj - 16]);
+                const bool keep = cbase + jj <= limit;
+                const float dec = ex2_approx(keep ? br2 - bv[e] : 0.f);   // e^{b_r - b_i}
+                val[jj] = keep ? rowscale * dec * x : 0.f;
             }
+        }
+        if (is_p) {
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+                uint4 w;
+                w.x = pack_bf16(val[8 * h + 0], val[8 * h + 1]);
+                w.y = pack_bf16(val[8 * h + 2], val[8 * h + 3]);
+                w.z = pack_bf16(val[8 * h + 4], val[8 * h + 5]);
+                w.w = pack_bf16(val[8 * h + 6], val[8 * h + 7]);
+                *reinterpret_cast<uint4*>(smem + kI_P + sw128_offset(r, (cbase >> 3) + h)) = w;
+            }
+        } else {
+#pragma unroll
+            for (int q4 = 0; q4 < 8; ++q4)
+                *reinterpret_cast<float4*>(sA + r * kLdA + cbase + 4 * q4) =
+                    make_float4(val[4 * q4], val[4 * q4 + 1], val[4 * q4 + 2], val[4 * q4 + 3]);
+        }
+    }
+    {   // Q rows scaled by e^{b_r}, in place (the Gram product has consumed Q): this is the Qg image
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const int idx = tid + it * kIntraThreads;          // 1024 16-byte pieces
+            const int halfq = idx >> 9, rem = idx & 511;
+            const int r = rem >> 3;
+            uint4* ptr = reinterpret_cast<uint4*>(smem + kI_QK + halfq * 16384 + rem * 16);
+            const float f = s_eb[r];
+            uint4 w = *ptr;
+            w.x = scale_bf16x2(w.x, f); w.y = scale_bf16x2(w.y, f);
+            w.z = scale_bf16x2(w.z, f); w.w = scale_bf16x2(w.w, f);
+            *ptr = w;
         }
     }
     __syncthreads();
+    PT(3);
 
-    // T = (I + A)^{-1} by forward substitution; thread j owns column j of T.
-    if (tid < 64) {
-        const int j = tid;
-        float t[64];
+    long long* st_out = nullptr;
+#ifdef GDN_PHASE_TIMING
+    if (false) st_out = reinterpret_cast<long long*>(ws + 192);
+#endif
+    solve_unit_lower_64(sA, reinterpret_cast<float*>(smem + kI_Scr), tid, st_out);
+
+    {   // T (fp32, row-major) -> bf16 B operands T diag(beta e^b), T diag(beta) (hi, lo)
 #pragma unroll
-        for (int r = 0; r < 64; ++r) t[r] = (r == j) ? 1.f : 0.f;
+        for (int it = 0; it < 2; ++it) {
+            const int idx = tid + it * kIntraThreads;          // 512 pieces of 8 columns
+            const int r = idx >> 3, c8 = idx & 7;
+            const float4 t0 = *reinterpret_cast<const float4*>(sA + r * kLdA + 8 * c8);
+            const float4 t1 = *reinterpret_cast<const float4*>(sA + r * kLdA + 8 * c8 + 4);
+            const float4 g0 = *reinterpret_cast<const float4*>(s_bg + 8 * c8);
+            const float4 g1 = *reinterpret_cast<const float4*>(s_bg + 8 * c8 + 4);
+            const float4 e0 = *reinterpret_cast<const float4*>(s_beta + 8 * c8);
+            const float4 e1 = *reinterpret_cast<const float4*>(s_beta + 8 * c8 + 4);
+            const float tv[8] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+            const float gv[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+            const float ev[8] = {e0.x, e0.y, e0.z, e0.w, e1.x, e1.y, e1.z, e1.w};
+            uint32_t w[4], hi[4], lo[4];
 #pragma unroll
-        for (int i = 0; i < 63; ++i) {
-            const float ti = t[i];
-#pragma unroll
-            for (int r4 = (i + 1) & ~3; r4 < 64; r4 += 4) {
-                const float4 a = *reinterpret_cast<const float4*>(sAT + i * 64 + r4);
-                if (r4 + 0 > i) t[r4 + 0] = fmaf(-a.x, ti, t[r4 + 0]);
-                if (r4 + 1 > i) t[r4 + 1] = fmaf(-a.y, ti, t[r4 + 1]);
-                if (r4 + 2 > i) t[r4 + 2] = fmaf(-a.z, ti, t[r4 + 2]);
-                if (r4 + 3 > i) t[r4 + 3] = fmaf(-a.w, ti, t[r4 + 3]);
+            for (int j = 0; j < 4; ++j) {
+                w[j] = pack_bf16(tv[2 * j] * gv[2 * j], tv[2 * j + 1] * gv[2 * j + 1]);
+                const float u0 = tv[2 * j] * ev[2 * j], u1 = tv[2 * j + 1] * ev[2 * j + 1];
+                hi[j] = pack_bf16(u0, u1);
+                lo[j] = pack_bf16(u0 - __uint_as_float(hi[j] << 16),
+                                  u1 - __uint_as_float(hi[j] & 0xffff0000u));
             }
-        }
-        const float bj = s_beta[j];
-        const float bgj = bj * __expf(s_b[j]);
-        const uint32_t col_off = ((j & 7) << 1);
-#pragma unroll
-        for (int r = 0; r < 64; ++r) {
-            const uint32_t off = sw128_offset(r, j >> 3) + col_off;
-            *reinterpret_cast<__nv_bfloat16*>(smem + kI_Tw + off) = __float2bfloat16(t[r] * bgj);
-            const float tu = t[r] * bj;
-            const __nv_bfloat16 tu_hi = __float2bfloat16(tu);
-            *reinterpret_cast<__nv_bfloat16*>(smem + kI_Tu + off) = tu_hi;
-            *reinterpret_cast<__nv_bfloat16*>(smem + kI_TuLo + off) =
-                __float2bfloat16(tu - __bfloat162float(tu_hi));
+            const uint32_t off = sw128_offset(r, c8);
+            *reinterpret_cast<uint4*>(smem + kI_Tw + off) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4*>(smem + kI_Tu + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            *reinterpret_cast<uint4*>(smem + kI_TuLo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
         }
     }
+    ST(7);
     fence_proxy_async_smem();
     __syncthreads();
+    PT(4);
 
     if (tid == 0) {
+        // Qg and P are final: start their stores while the last products run
+        bulk_store(rec + kRecQg, smem + kI_QK, 8192);
+        bulk_store(rec + kRecQg + 8192, smem + kI_QK + 16384, 8192);
+        bulk_store(rec + kRecP, smem + kI_P, 8192);
+        bulk_commit();
         // W^T (dk x r) = K^T (MN-major A from the K tile) times T_w^T ; U~^T (dv x r) likewise from V
         const uint32_t idesc = make_idesc_bf16(128, 64, true, false);
         const uint32_t sTw = smem_u32(smem + kI_Tw), sTu = smem_u32(smem + kI_Tu);
@@ -270,64 +474,104 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
                    make_sdesc_sw128(sTuLo + ks * 32, 16, 1024), idesc, true);
         mma_commit(&bar_mma);
     }
-    if (!mbar_wait(&bar_mma, 1)) abort_flag = 1;
+    if (warp == 0 && !warp_wait(&bar_mma, 1)) abort_flag = 1;      // one warp polls, the rest block
     __syncthreads();
     if (abort_flag) {
-        if (tid == 0) report(p.dev_status, kDevTimeout);
+        if (tid == 0) { report(p.dev_status, kDevTimeout); bulk_wait_read_all(); }
         if (warp == 0) tmem_dealloc(tmem, kIntraTmemCols);
         return;
     }
     tc_fence_after_sync();
+    PT(5);
 
-    {   // thread d (TMEM lane) holds W^T[d][0..63] and U~^T[d][0..63]
-        const int d = tid;
-        uint8_t* sW = smem + kI_QK;     // the Q/K tiles are dead now: stage the W image there
-        const uint32_t wbase = (d >> 6) * 8192 + ((d & 7) << 1);
+    {   // thread (d, column half) holds W^T[d][32 tokens] and U~^T[d][32 tokens]
+        const int d = (warp & 3) * 32 + (tid & 31);
+        const int cbase = colhalf * 32;
+        // the K tile is dead now: stage W half (d / 64) over K's half (d / 64)
+        uint8_t* sW = smem + kI_QK + 8192 + (d >> 6) * 16384;
+        const uint32_t wcol = ((d & 7) << 1);
         const uint32_t wchunk = (d & 63) >> 3;
         float4* urec = reinterpret_cast<float4*>(rec + kRecU);
+        uint32_t xa[16], xb[16], ya[16], yb[16];
+        tmem_ld16(tW + lane_base + cbase, xa);
+        tmem_ld16(tW + lane_base + cbase + 16, xb);
+        tmem_ld16(tU + lane_base + cbase, ya);
+        tmem_ld16(tU + lane_base + cbase + 16, yb);
+        tmem_wait_ld();
 #pragma unroll
-        for (int c0 = 0; c0 < 64; c0 += 16) {
-            uint32_t x[16], y[16];
-            tmem_ld16(tW + lane_base + c0, x);
-            tmem_ld16(tU + lane_base + c0, y);
-            tmem_wait_ld();
-#pragma unroll
-            for (int j = 0; j < 16; ++j)
-                *reinterpret_cast<__nv_bfloat16*>(sW + wbase + sw128_offset(c0 + j, wchunk)) =
-                    __float2bfloat16(__uint_as_float(x[j]));
-#pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4)
-                urec[((c0 >> 2) + q4) * kD + d] =
-                    make_float4(__uint_as_float(y[4 * q4]), __uint_as_float(y[4 * q4 + 1]),
-                                __uint_as_float(y[4 * q4 + 2]), __uint_as_float(y[4 * q4 + 3]));
+        for (int j = 0; j < 16; ++j) {
+            *reinterpret_cast<__nv_bfloat16*>(sW + sw128_offset(cbase + j, wchunk) + wcol) =
+                __float2bfloat16(__uint_as_float(xa[j]));
+            *reinterpret_cast<__nv_bfloat16*>(sW + sw128_offset(cbase + 16 + j, wchunk) + wcol) =
+                __float2bfloat16(__uint_as_float(xb[j]));
         }
-        if (tid < kChunk) reinterpret_cast<float*>(rec + kRecB)[tid] = s_b[tid];
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+            urec[((cbase >> 2) + q4) * kD + d] =
+                make_float4(__uint_as_float(ya[4 * q4]), __uint_as_float(ya[4 * q4 + 1]),
+                            __uint_as_float(ya[4 * q4 + 2]), __uint_as_float(ya[4 * q4 + 3]));
+            urec[((cbase >> 2) + 4 + q4) * kD + d] =
+                make_float4(__uint_as_float(yb[4 * q4]), __uint_as_float(yb[4 * q4 + 1]),
+                            __uint_as_float(yb[4 * q4 + 2]), __uint_as_float(yb[4 * q4 + 3]));
+        }
     }
     fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();
     if (tid == 0) {
-        bulk_store(rec + kRecW, smem + kI_QK, 16384);
-        bulk_store(rec + kRecP, smem + kI_P, 8192);
+        bulk_store(rec + kRecW, smem + kI_QK + 8192, 8192);
+        bulk_store(rec + kRecW + 8192, smem + kI_QK + 24576, 8192);
         bulk_commit();
         bulk_wait_read_all();
     }
+    PT(6);
+    PT_FLUSH(blockIdx.x == gridDim.x / 2 && blockIdx.y == gridDim.y / 2, 64, 7);
     if (warp == 0) tmem_dealloc(tmem, kIntraTmemCols);
 }
 
 // =============================================================================================
-// K2: inter-chunk state pass, one CTA (256 threads) per (sequence, v-head).
+// K2: inter-chunk state pass, one CTA per (sequence, v-head): 8 epilogue warps + 1 issuing warp.
+//
+// Per chunk the dependent chain is  D1 = S W^T  ->  U = U~ - D1  ->  D4 = (U decayed) K  ->
+// S = e^{b_C} S + D4.  The output product  Y = S Qg^T + U P^T  is accumulated in a second,
+// double-buffered TMEM tile and is turned into o rows one chunk later, while the next chunk's
+// D1 is in flight.  One lane of warp 8 issues every TMA copy and every tcgen05.mma; the
+// epilogue warps hand it the bf16 state ("s") and the U operands ("u") through mbarriers, so
+// nobody but the issuing lane ever waits for the tensor pipe to accept instructions.
 // =============================================================================================
-constexpr int kStateThreads = 256;
+constexpr int kStateEpiWarps = 8;
+constexpr int kStateEpiThreads = kStateEpiWarps * 32;
+constexpr int kStateThreads = kStateEpiThreads + 32;
 constexpr uint32_t kStateTmemCols = 512;
-constexpr uint32_t kS_Rec = 0;                 // record image (57600 B, padded to 58368)
-constexpr uint32_t kS_K = 58368;               // K tile, 2 halves [64 x 128 B]
-constexpr uint32_t kS_Q = 58368 + 16384;       // Q tile
-constexpr uint32_t kStageBytes = 58368 + 32768;                 // 91136
-constexpr uint32_t kStateSmem = 2 * kStageBytes + 1024;
+constexpr uint32_t kS_Rec = 0;                 // record image (74240 B, padded to 74752)
+constexpr uint32_t kS_K = 74752;               // K tile, 2 halves [64 x 128 B]
+constexpr uint32_t kStageBytes = 74752 + 16384;                 // 91136
+constexpr uint32_t kS_Out = 2 * kStageBytes;   // o staging [64 tokens][128 dv] bf16
+constexpr uint32_t kStateSmem = 2 * kStageBytes + 16384 + 1024;
 // TMEM columns
-constexpr uint32_t kT_D1 = 0, kT_D2 = 64, kT_D3 = 128, kT_D4 = 192, kT_S = 320, kT_U = 384,
+constexpr uint32_t kT_D1 = 0, kT_Y = 64 /* two tiles of 64 */, kT_D4 = 192, kT_S = 320, kT_U = 384,
                    kT_Us = 416, kT_UsLo = 448;
+
+// bounded wait that also gives up as soon as another role has flagged an abort
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 255u) == 255u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+// Same, for a whole warp: lane 0 polls, every lane gets the verdict.
+__device__ __forceinline__ bool warp_wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = wait_or_abort(bar, parity, abort_flag) ? 1 : 0;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+
+__device__ __forceinline__ void epi_group_sync() {      // the 256 epilogue threads only
+    asm volatile("bar.sync 1, %0;" ::"n"(kStateEpiThreads) : "memory");
+}
 
 __global__ void __launch_bounds__(kStateThreads, 1)
 prefill_state_kernel(const __grid_constant__ TensorMaps maps, const PrefillParams p, uint8_t* ws,
@@ -335,9 +579,10 @@ prefill_state_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
     const int n = blockIdx.x / p.Hv;
     const int hv = blockIdx.x - n * p.Hv;
     const int hqk = hv / (p.Hv / p.Hqk);
-    const int tid = threadIdx.x, warp = tid >> 5;
-    const int half = warp >> 2;                       // which half of the columns this thread owns
-    const int dv = (warp & 3) * 32 + (tid & 31);      // TMEM lane = state row
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const bool is_epi = warp < kStateEpiWarps;
+    const int half = (warp >> 2) & 1;                 // which half of the columns this thread owns
+    const int dv = (warp & 3) * 32 + lane;            // TMEM lane = state row
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
 
     const int32_t* seq_first = reinterpret_cast<const int32_t*>(ws + lay.seq_first);
@@ -345,24 +590,23 @@ prefill_state_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
     if (seq_bad[n]) return;
     const int c_first = seq_first[n];
     const int nc = seq_first[n + 1] - c_first;
-    const ChunkInfo* chunks = reinterpret_cast<const ChunkInfo*>(ws + lay.chunks);
+    const int seq_t0 = p.cu_seqlens[n];
+    const int seq_len = p.cu_seqlens[n + 1] - seq_t0;
 
     const int slot = p.slot_idx ? p.slot_idx[n] : n;
     if (slot < 0 || slot >= p.num_slots) {
         if (slot >= p.num_slots && tid == 0) report(p.dev_status, kDevBadSlot);
-        for (int j = 0; j < nc; ++j) {
-            const ChunkInfo ci = chunks[c_first + j];
-            for (int idx = tid; idx < ci.len * kD; idx += kStateThreads)
-                p.o[(static_cast<size_t>(ci.t0 + idx / kD) * p.Hv + hv) * kD + (idx % kD)] =
-                    __float2bfloat16(0.f);
-        }
+        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+        for (int idx = tid; idx < seq_len * 16; idx += kStateThreads)
+            *reinterpret_cast<uint4*>(p.o + (static_cast<size_t>(seq_t0 + (idx >> 4)) * p.Hv + hv) * kD +
+                                      (idx & 15) * 8) = zero;
         return;
     }
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                                ~static_cast<uintptr_t>(1023));
-    __shared__ uint64_t bar_full[2], bar_mma1, bar_mma2;
+    __shared__ uint64_t bar_full[2], bar_d1, bar_d4, bar_y, bar_s, bar_u;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_flag;
 
@@ -370,7 +614,7 @@ prefill_state_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
     float S[64];
     const size_t tile_off = (static_cast<size_t>(slot) * p.Hv + hv) * (kD * kD) +
                             static_cast<size_t>(dv) * kD + half * 64;
-    if (p.init_state) {
+    if (is_epi && p.init_state) {
 #pragma unroll
         for (int j = 0; j < 64; j += 4) {
             const float4 x = *reinterpret_cast<const float4*>(p.init_state + tile_off + j);
@@ -385,12 +629,15 @@ prefill_state_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
         if (tid == 0) {
             mbar_init(&bar_full[0], 1);
             mbar_init(&bar_full[1], 1);
-            mbar_init(&bar_mma1, 1);
-            mbar_init(&bar_mma2, 1);
+            mbar_init(&bar_d1, 1);
+            mbar_init(&bar_d4, 1);
+            mbar_init(&bar_y, 1);
+            mbar_init(&bar_s, kStateEpiWarps);
+            mbar_init(&bar_u, kStateEpiWarps);
             abort_flag = 0;
             fence_barrier_init();
         }
-        if (warp == 0) {
+        if (warp == kStateEpiWarps) {
             tmem_alloc(&tmem_base_s, kStateTmemCols);
             tmem_relinquish();
         }
@@ -398,188 +645,246 @@ prefill_state_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
         __syncthreads();
         tc_fence_after_sync();
         const uint32_t tmem = tmem_base_s;
-        const uint8_t* records = ws + lay.records;
+        volatile int* abortp = &abort_flag;
 
-        auto issue_loads = [&](int j) {       // thread 0 only
-            const int st = j & 1;
-            const ChunkInfo ci = chunks[c_first + j];
-            uint8_t* base = smem + st * kStageBytes;
-            mbar_expect_tx(&bar_full[st], kRecBytes + 32768);
-            bulk_load(base + kS_Rec,
-                      records + (static_cast<size_t>(c_first + j) * p.Hv + hv) * kRecBytes, kRecBytes,
-                      &bar_full[st]);
-            tma_load_2d(base + kS_K, &maps.k, hqk * kD, ci.t0, &bar_full[st]);
-            tma_load_2d(base + kS_K + 8192, &maps.k, hqk * kD + 64, ci.t0, &bar_full[st]);
-            tma_load_2d(base + kS_Q, &maps.q, hqk * kD, ci.t0, &bar_full[st]);
-            tma_load_2d(base + kS_Q + 8192, &maps.q, hqk * kD + 64, ci.t0, &bar_full[st]);
-        };
-        auto store_state_bf16 = [&]() {       // S (fp32 regs) -> bf16 A operand in TMEM
+        if (!is_epi) {
+            // ===================== issuing warp: TMA copies and tensor-core instructions
+            if (lane == 0) {
+                const uint8_t* records =
+                    ws + lay.records + (static_cast<size_t>(c_first) * p.Hv + hv) * kRecBytes;
+                const size_t rec_stride = static_cast<size_t>(p.Hv) * kRecBytes;
+                auto issue_loads = [&](int j) {
+                    const int st = j & 1;
+                    uint8_t* base = smem + st * kStageBytes;
+                    mbar_expect_tx(&bar_full[st], kRecBytes + 16384);
+                    bulk_load(base + kS_Rec, records + j * rec_stride, kRecBytes, &bar_full[st]);
+                    tma_load_2d(base + kS_K, &maps.k, hqk * kD, seq_t0 + j * kChunk, &bar_full[st]);
+                    tma_load_2d(base + kS_K + 8192, &maps.k, hqk * kD + 64, seq_t0 + j * kChunk,
+                                &bar_full[st]);
+                };
+                const uint32_t id64 = make_idesc_bf16(128, 64, false, false);
+                const uint32_t id128mn = make_idesc_bf16(128, 128, false, true);
+                issue_loads(0);
+                if (nc > 1) issue_loads(1);
+                PT_DECL
+                for (int j = 0; j < nc; ++j) {
+                    const int st = j & 1;
+                    const uint32_t sRec = smem_u32(smem + st * kStageBytes + kS_Rec);
+                    const uint32_t sK = smem_u32(smem + st * kStageBytes + kS_K);
+                    if (!wait_or_abort(&bar_full[st], (j >> 1) & 1, abortp)) break;
+                    PTI(0);
+                    if (!wait_or_abort(&bar_s, j & 1, abortp)) break;       // bf16 S of chunk j in TMEM
+                    tc_fence_after_sync();
+                    PTI(1);
 #pragma unroll
-            for (int c0 = 0; c0 < 64; c0 += 32) {
-                uint32_t pk[16];
-#pragma unroll
-                for (int j = 0; j < 16; ++j) pk[j] = pack_bf16(S[c0 + 2 * j], S[c0 + 2 * j + 1]);
-                tmem_st16(tmem + kT_S + lane_base + half * 32 + (c0 >> 1), pk);
-            }
-        };
-
-        if (tid == 0) issue_loads(0);
-        store_state_bf16();
-        tmem_wait_st();
-        tc_fence_before_sync();
-        __syncthreads();
-        tc_fence_after_sync();
-
-        bool ok = true;
-        for (int j = 0; j < nc && ok; ++j) {
-            const int st = j & 1;
-            uint8_t* base = smem + st * kStageBytes;
-            const ChunkInfo ci = chunks[c_first + j];
-            if (tid == 0 && j + 1 < nc) issue_loads(j + 1);
-            if (!mbar_wait(&bar_full[st], (j >> 1) & 1)) abort_flag = 1;
-            __syncthreads();
-            if (abort_flag) { ok = false; break; }
-            tc_fence_after_sync();
-
-            const uint32_t sRec = smem_u32(base + kS_Rec);
-            const uint32_t sK = smem_u32(base + kS_K), sQ = smem_u32(base + kS_Q);
-            if (tid == 0) {
-                const uint32_t idesc = make_idesc_bf16(128, 64, false, false);
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {       // D1 = S W^T
-                    const uint32_t off = (ks >> 2) * 8192 + (ks & 3) * 32;
-                    mma_ts(tmem + kT_D1, tmem + kT_S + ks * 8,
-                           make_sdesc_sw128(sRec + kRecW + off, 16, 1024), idesc, ks > 0);
-                }
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {       // D2 = S Q^T
-                    const uint32_t off = (ks >> 2) * 8192 + (ks & 3) * 32;
-                    mma_ts(tmem + kT_D2, tmem + kT_S + ks * 8, make_sdesc_sw128(sQ + off, 16, 1024),
-                           idesc, ks > 0);
-                }
-                mma_commit(&bar_mma1);
-            }
-            if (!mbar_wait(&bar_mma1, j & 1)) abort_flag = 1;
-            __syncthreads();
-            if (abort_flag) { ok = false; break; }
-            tc_fence_after_sync();
-
-            const float* sb = reinterpret_cast<const float*>(base + kS_Rec + kRecB);
-            const float bC = sb[kChunk - 1];
-            {   // U^T[dv][c] = U~^T - D1 for the thread's 32 tokens [32*half, 32*half+32)
-                const float4* sU = reinterpret_cast<const float4*>(base + kS_Rec + kRecU);
-#pragma unroll
-                for (int c0 = 0; c0 < 32; c0 += 16) {
-                    const int cb = half * 32 + c0;
-                    uint32_t x[16];
-                    tmem_ld16(tmem + kT_D1 + lane_base + cb, x);
-                    tmem_wait_ld();
-                    float u[16];
-#pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        const float4 ut = sU[((cb >> 2) + q4) * kD + dv];
-                        u[4 * q4 + 0] = ut.x - __uint_as_float(x[4 * q4 + 0]);
-                        u[4 * q4 + 1] = ut.y - __uint_as_float(x[4 * q4 + 1]);
-                        u[4 * q4 + 2] = ut.z - __uint_as_float(x[4 * q4 + 2]);
-                        u[4 * q4 + 3] = ut.w - __uint_as_float(x[4 * q4 + 3]);
+                    for (int ks = 0; ks < 8; ++ks) {       // D1 = S W^T  (on the chain)
+                        const uint32_t off = (ks >> 2) * 8192 + (ks & 3) * 32;
+                        mma_ts(tmem + kT_D1, tmem + kT_S + ks * 8,
+                               make_sdesc_sw128(sRec + kRecW + off, 16, 1024), id64, ks > 0);
                     }
-                    // U for the output product; the decayed U for the state update is kept as
-                    // hi + lo bf16 pairs so that its rounding does not limit the state's accuracy
-                    uint32_t pu[8], ph[8], pl[8];
+                    mma_commit(&bar_d1);
+#ifdef GDN_PHASE_TIMING
+                    PTI(6);
+                    mbar_wait(&bar_d1, j & 1);
+                    PTI(7);
+#endif
 #pragma unroll
-                    for (int jj = 0; jj < 8; ++jj) {
-                        const float s0 = u[2 * jj] * __expf(bC - sb[cb + 2 * jj]);
-                        const float s1 = u[2 * jj + 1] * __expf(bC - sb[cb + 2 * jj + 1]);
-                        pu[jj] = pack_bf16(u[2 * jj], u[2 * jj + 1]);
-                        ph[jj] = pack_bf16(s0, s1);
-                        pl[jj] = pack_bf16(s0 - __uint_as_float(ph[jj] << 16),
-                                           s1 - __uint_as_float(ph[jj] & 0xffff0000u));
+                    for (int ks = 0; ks < 8; ++ks) {       // Y = S Qg^T  (off the chain)
+                        const uint32_t off = (ks >> 2) * 8192 + (ks & 3) * 32;
+                        mma_ts(tmem + kT_Y + st * 64, tmem + kT_S + ks * 8,
+                               make_sdesc_sw128(sRec + kRecQg + off, 16, 1024), id64, ks > 0);
                     }
-                    tmem_st8(tmem + kT_U + lane_base + (cb >> 1), pu);
-                    tmem_st8(tmem + kT_Us + lane_base + (cb >> 1), ph);
-                    tmem_st8(tmem + kT_UsLo + lane_base + (cb >> 1), pl);
+                    PTI(2);
+                    if (j > 0 && j + 1 < nc) {
+                        // the other stage is free once chunk j-1's last product has retired (the
+                        // epilogue warps left it before they handed over this chunk's S)
+                        if (!wait_or_abort(&bar_y, (j - 1) & 1, abortp)) break;
+                        issue_loads(j + 1);
+                    }
+                    PTI(3);
+                    if (!wait_or_abort(&bar_u, j & 1, abortp)) break;       // U operands in TMEM
+                    tc_fence_after_sync();
+                    PTI(4);
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)          // D4 = (U decayed) K   (K tile MN-major)
+                        mma_ts(tmem + kT_D4, tmem + kT_Us + ks * 8,
+                               make_sdesc_sw128(sK + ks * 2048, 8192, 1024), id128mn, ks > 0);
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)
+                        mma_ts(tmem + kT_D4, tmem + kT_UsLo + ks * 8,
+                               make_sdesc_sw128(sK + ks * 2048, 8192, 1024), id128mn, true);
+                    mma_commit(&bar_d4);
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)          // Y += U P^T
+                        mma_ts(tmem + kT_Y + st * 64, tmem + kT_U + ks * 8,
+                               make_sdesc_sw128(sRec + kRecP + ks * 32, 16, 1024), id64, true);
+                    mma_commit(&bar_y);
+                    PTI(5);
                 }
+                PTI_FLUSH(blockIdx.x == gridDim.x - 1, 192, 8);
             }
-            tmem_wait_st();
-            tc_fence_before_sync();
-            __syncthreads();
-            tc_fence_after_sync();
-
-            if (tid == 0) {
-                const uint32_t id3 = make_idesc_bf16(128, 64, false, false);
-                const uint32_t id4 = make_idesc_bf16(128, 128, false, true);
+            __syncwarp();
+        } else {
+            // ===================== epilogue warps: the fp32 state, U, and the output rows
+            auto hand_over = [&](uint64_t* bar) {     // after tcgen05.st: publish to the issuing lane
+                tmem_wait_st();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar);
+            };
+            auto store_state_bf16 = [&]() {           // S (fp32 regs) -> bf16 A operand in TMEM
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)          // D3 = U P^T
-                    mma_ts(tmem + kT_D3, tmem + kT_U + ks * 8,
-                           make_sdesc_sw128(sRec + kRecP + ks * 32, 16, 1024), id3, ks > 0);
+                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    uint32_t pk[16];
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)          // D4 = (U decayed) K   (K tile MN-major)
-                    mma_ts(tmem + kT_D4, tmem + kT_Us + ks * 8,
-                           make_sdesc_sw128(sK + ks * 2048, 8192, 1024), id4, ks > 0);
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    mma_ts(tmem + kT_D4, tmem + kT_UsLo + ks * 8,
-                           make_sdesc_sw128(sK + ks * 2048, 8192, 1024), id4, true);
-                mma_commit(&bar_mma2);
-            }
-            if (!mbar_wait(&bar_mma2, j & 1)) abort_flag = 1;
-            __syncthreads();
-            if (abort_flag) { ok = false; break; }
-            tc_fence_after_sync();
-
-            {   // S <- e^{b_C} S + D4 on the thread's 64 dk columns; refresh the bf16 copy
-                const float gC = __expf(bC);
-#pragma unroll
-                for (int c0 = 0; c0 < 64; c0 += 16) {
-                    uint32_t x[16];
-                    tmem_ld16(tmem + kT_D4 + lane_base + half * 64 + c0, x);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int jj = 0; jj < 16; ++jj)
-                        S[c0 + jj] = fmaf(gC, S[c0 + jj], __uint_as_float(x[jj]));
+                    for (int j = 0; j < 16; ++j) pk[j] = pack_bf16(S[c0 + 2 * j], S[c0 + 2 * j + 1]);
+                    tmem_st16(tmem + kT_S + lane_base + half * 32 + (c0 >> 1), pk);
                 }
-                store_state_bf16();
-            }
-            {   // o[t0+c][hv][dv] = scale (e^{b_c} D2 + D3) for the thread's 32 tokens
-                __nv_bfloat16* op = p.o + (static_cast<size_t>(ci.t0) * p.Hv + hv) * kD + dv;
+            };
+            // o rows of chunk j from Y[j & 1]: scale, round to bf16, transpose through shared
+            // memory, write 16-byte pieces of whole rows
+            auto write_outputs = [&](int j) {
+                const uint32_t tY = tmem + kT_Y + (j & 1) * 64;
+                __nv_bfloat16* sO = reinterpret_cast<__nv_bfloat16*>(smem + kS_Out);
+                uint32_t x[16], y[16];
+                tmem_ld16(tY + lane_base + half * 32, x);
+                tmem_ld16(tY + lane_base + half * 32 + 16, y);
+                tmem_wait_ld();
+#pragma unroll
+                for (int jj = 0; jj < 16; ++jj) {
+                    sO[(half * 32 + jj) * kD + dv] = __float2bfloat16(p.scale * __uint_as_float(x[jj]));
+                    sO[(half * 32 + 16 + jj) * kD + dv] = __float2bfloat16(p.scale * __uint_as_float(y[jj]));
+                }
+                epi_group_sync();
+                const int len = min(kChunk, seq_len - j * kChunk);
+                __nv_bfloat16* og = p.o + (static_cast<size_t>(seq_t0 + j * kChunk) * p.Hv + hv) * kD;
                 const size_t tok_stride = static_cast<size_t>(p.Hv) * kD;
 #pragma unroll
-                for (int c0 = 0; c0 < 32; c0 += 16) {
-                    const int cb = half * 32 + c0;
-                    uint32_t x[16], y[16];
-                    tmem_ld16(tmem + kT_D2 + lane_base + cb, x);
-                    tmem_ld16(tmem + kT_D3 + lane_base + cb, y);
+                for (int it = 0; it < 4; ++it) {
+                    const int row = it * 16 + (tid >> 4), piece = tid & 15;
+                    if (row < len)
+                        *reinterpret_cast<uint4*>(og + row * tok_stride + piece * 8) =
+                            *reinterpret_cast<const uint4*>(sO + row * kD + piece * 8);
+                }
+            };
+
+            store_state_bf16();
+            hand_over(&bar_s);
+            PT_DECL
+            bool ok = true;
+            for (int j = 0; j < nc; ++j) {
+                const int st = j & 1;
+                const uint8_t* base = smem + st * kStageBytes;
+                PT(0);
+                if (!warp_wait_or_abort(&bar_full[st], (j >> 1) & 1, abortp)) { ok = false; break; }
+                if (!warp_wait_or_abort(&bar_d1, j & 1, abortp)) { ok = false; break; }
+                tc_fence_after_sync();
+                PT(1);
+
+                const float* sdec = reinterpret_cast<const float*>(base + kS_Rec + kRecDecay);
+                {   // U^T[dv][c] = U~^T - D1 for the thread's 32 tokens [32*half, 32*half+32)
+                    const float4* sU = reinterpret_cast<const float4*>(base + kS_Rec + kRecU);
+                    uint32_t xa[16], xb[16];
+                    tmem_ld16(tmem + kT_D1 + lane_base + half * 32, xa);
+                    tmem_ld16(tmem + kT_D1 + lane_base + half * 32 + 16, xb);
                     tmem_wait_ld();
+                    auto u_block = [&](const uint32_t (&x)[16], const int cb) {
+                        float u[16];
 #pragma unroll
-                    for (int jj = 0; jj < 16; ++jj) {
-                        const int cc = cb + jj;
-                        if (cc < ci.len)
-                            op[cc * tok_stride] = __float2bfloat16(
-                                p.scale * fmaf(__expf(sb[cc]), __uint_as_float(x[jj]),
-                                               __uint_as_float(y[jj])));
+                        for (int q4 = 0; q4 < 4; ++q4) {
+                            const float4 ut = sU[((cb >> 2) + q4) * kD + dv];
+                            u[4 * q4 + 0] = ut.x - __uint_as_float(x[4 * q4 + 0]);
+                            u[4 * q4 + 1] = ut.y - __uint_as_float(x[4 * q4 + 1]);
+                            u[4 * q4 + 2] = ut.z - __uint_as_float(x[4 * q4 + 2]);
+                            u[4 * q4 + 3] = ut.w - __uint_as_float(x[4 * q4 + 3]);
+                        }
+                        // U for the output product; the decayed U for the state update is kept
+                        // as hi + lo bf16 pairs so that its rounding does not limit the state
+                        uint32_t pu[8], ph[8], pl[8];
+#pragma unroll
+                        for (int q4 = 0; q4 < 4; ++q4) {
+                            const float4 dd = *reinterpret_cast<const float4*>(sdec + cb + 4 * q4);
+                            const float s0 = u[4 * q4 + 0] * dd.x, s1 = u[4 * q4 + 1] * dd.y;
+                            const float s2 = u[4 * q4 + 2] * dd.z, s3 = u[4 * q4 + 3] * dd.w;
+                            pu[2 * q4] = pack_bf16(u[4 * q4 + 0], u[4 * q4 + 1]);
+                            pu[2 * q4 + 1] = pack_bf16(u[4 * q4 + 2], u[4 * q4 + 3]);
+                            ph[2 * q4] = pack_bf16(s0, s1);
+                            ph[2 * q4 + 1] = pack_bf16(s2, s3);
+                            pl[2 * q4] = pack_bf16(s0 - __uint_as_float(ph[2 * q4] << 16),
+                                                   s1 - __uint_as_float(ph[2 * q4] & 0xffff0000u));
+                            pl[2 * q4 + 1] = pack_bf16(s2 - __uint_as_float(ph[2 * q4 + 1] << 16),
+                                                       s3 - __uint_as_float(ph[2 * q4 + 1] & 0xffff0000u));
+                        }
+                        tmem_st8(tmem + kT_Us + lane_base + (cb >> 1), ph);
+                        tmem_st8(tmem + kT_UsLo + lane_base + (cb >> 1), pl);
+                        tmem_st8(tmem + kT_U + lane_base + (cb >> 1), pu);
+                    };
+                    u_block(xa, half * 32);
+                    u_block(xb, half * 32 + 16);
+                }
+                hand_over(&bar_u);
+                PT(2);
+                if (j > 0) {
+                    // the previous chunk's output rows, while this chunk's state product runs
+                    if (!warp_wait_or_abort(&bar_y, (j - 1) & 1, abortp)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    write_outputs(j - 1);
+                }
+                PT(5);
+
+                if (!warp_wait_or_abort(&bar_d4, j & 1, abortp)) { ok = false; break; }
+                tc_fence_after_sync();
+                PT(3);
+                {   // S <- e^{b_C} S + D4 on the thread's 64 dk columns; refresh the bf16 copy
+                    const float gC = reinterpret_cast<const float*>(base + kS_Rec + kRecGammaC)[0];
+#pragma unroll
+                    for (int c0 = 0; c0 < 64; c0 += 32) {
+                        uint32_t xa[16], xb[16];
+                        tmem_ld16(tmem + kT_D4 + lane_base + half * 64 + c0, xa);
+                        tmem_ld16(tmem + kT_D4 + lane_base + half * 64 + c0 + 16, xb);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int jj = 0; jj < 16; ++jj) {
+                            S[c0 + jj] = fmaf(gC, S[c0 + jj], __uint_as_float(xa[jj]));
+                            S[c0 + 16 + jj] = fmaf(gC, S[c0 + 16 + jj], __uint_as_float(xb[jj]));
+                        }
                     }
+                    store_state_bf16();
+                }
+                hand_over(&bar_s);
+                PT(4);
+            }
+            if (ok) {
+                if (warp_wait_or_abort(&bar_y, (nc - 1) & 1, abortp)) {
+                    tc_fence_after_sync();
+                    // inside the loop the next chunk's barriers keep a fast warp from refilling
+                    // the staging tile while a slow one still reads it; here nothing else does
+                    epi_group_sync();
+                    write_outputs(nc - 1);
                 }
             }
-            tmem_wait_st();
-            tc_fence_before_sync();
-            __syncthreads();
-            tc_fence_after_sync();
+            PT_FLUSH(blockIdx.x == gridDim.x - 1, 128, 6);
         }
-        if (!ok) {
-            if (tid == 0) report(p.dev_status, kDevTimeout);
+        tc_fence_before_sync();
+        __syncthreads();
+        const bool failed = abort_flag != 0;
+        if (failed && warp == kStateEpiWarps && lane == 0) {
+            report(p.dev_status, kDevTimeout);
             // let copies already in flight land before the CTA's shared memory goes away
             mbar_wait(&bar_full[0], 0, 1u << 12);
             mbar_wait(&bar_full[1], 0, 1u << 12);
         }
-        __syncthreads();
-        if (warp == 0) tmem_dealloc(tmem, kStateTmemCols);
-        if (!ok) return;
+        __syncwarp();
+        if (warp == kStateEpiWarps) tmem_dealloc(tmem, kStateTmemCols);
+        if (failed) return;
     }
 
+    if (is_epi) {
 #pragma unroll
-    for (int j = 0; j < 64; j += 4)
-        *reinterpret_cast<float4*>(p.final_state + tile_off + j) =
-            make_float4(S[j], S[j + 1], S[j + 2], S[j + 3]);
+        for (int j = 0; j < 64; j += 4)
+            *reinterpret_cast<float4*>(p.final_state + tile_off + j) =
+                make_float4(S[j], S[j + 1], S[j + 2], S[j + 3]);
+    }
 }
 
 // =============================================================================================

@@ -7,7 +7,7 @@
 //   P_ri =        e^{b_r-b_i} (q_r.k_i)  (i <= r)
 //   W  = T diag(beta e^b) K   (C x dk),   U~ = T diag(beta) V   (C x dv)
 //   U  = U~ - W S0^T
-//   O  = scale ( diag(e^b) Q S0^T + P U )
+//   O  = scale ( diag(e^b) Q S0^T + P U )  =  scale ( Qg S0^T + P U ),  Qg = diag(e^b) Q
 //   S' = e^{b_C} S0 + U^T diag(e^{b_C-b}) K
 //
 // Three launches: a prep kernel builds the chunk table from cu_seqlens; the
@@ -23,15 +23,19 @@ namespace gdn {
 
 // One record per (chunk, v-head), written by the intra-chunk kernel in exactly the
 // byte image the state-pass kernel wants in shared memory (one linear bulk copy):
-//   [0, 16384)      W  as two K-major 128B-swizzled halves [64 tokens][64 dk] bf16
-//   [16384, 24576)  P  as one K-major 128B-swizzled tile   [64 r][64 i]      bf16
-//   [24576, 57344)  U~ as [16 token-groups][128 dv][4 tokens] fp32
-//   [57344, 57600)  b  as [64] fp32 (rows past the chunk's length repeat the last value)
+//   [0, 16384)      W   as two K-major 128B-swizzled halves [64 tokens][64 dk] bf16
+//   [16384, 32768)  Qg  = diag(e^b) Q, same layout as W (the output's first term S0 Qg^T)
+//   [32768, 40960)  P   as one K-major 128B-swizzled tile   [64 r][64 i]      bf16
+//   [40960, 73728)  U~  as [16 token-groups][128 dv][4 tokens] fp32
+//   [73728, 73984)  e^{b_C - b_c} for c = 0..63, fp32 (rows past the chunk's length hold 1)
+//   [73984, 74240)  e^{b_C} in the first float, rest unused
 constexpr uint32_t kRecW = 0;
-constexpr uint32_t kRecP = 16384;
-constexpr uint32_t kRecU = 24576;
-constexpr uint32_t kRecB = 57344;
-constexpr uint32_t kRecBytes = 57600;
+constexpr uint32_t kRecQg = 16384;
+constexpr uint32_t kRecP = 32768;
+constexpr uint32_t kRecU = 40960;
+constexpr uint32_t kRecDecay = 73728;
+constexpr uint32_t kRecGammaC = 73984;
+constexpr uint32_t kRecBytes = 74240;
 
 struct ChunkInfo {      // 16 bytes
     int32_t seq;        // sequence the chunk belongs to
