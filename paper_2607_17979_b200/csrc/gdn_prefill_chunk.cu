@@ -100,8 +100,8 @@ constexpr uint32_t kI_Tu = 57344;      // T diag(beta) rounded to bf16 ...
 constexpr uint32_t kI_TuLo = 65536;    // ... and the bf16 remainder (hi + lo carries ~16 bits)
 constexpr uint32_t kI_P = 73728;       // P image staging
 constexpr uint32_t kI_A = 81920;       // A, then T in place: fp32 [64][kLdA]
-constexpr uint32_t kI_Scr = kI_A + 64 * kLdA * 4;      // solve scratch, fp32 [32][36]
-constexpr uint32_t kI_End = kI_Scr + 32 * 36 * 4;
+constexpr uint32_t kI_Scr = kI_A + 64 * kLdA * 4;      // solve scratch, fp32 [32][40]
+constexpr uint32_t kI_End = kI_Scr + 32 * 40 * 4;
 constexpr uint32_t kIntraSmem = kI_End + 1024;         // + alignment slack
 
 struct TensorMaps {
@@ -114,11 +114,51 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
+// One 16x8 output tile  C += A[16 x 8*ksteps] * B[8*ksteps x 8]  on mma.sync m16n8k8 with both
+// operands split into tf32 hi + lo parts (three products; the lo*lo term is dropped), which keeps
+// fp32-level accuracy.  A, B: fp32 row-major in shared memory; g = lane / 4, t = lane % 4.
+__device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo) {
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(hi) : "f"(x));
+    const float rem = x - __uint_as_float(hi);
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(lo) : "f"(rem));
+}
+__device__ __forceinline__ void mma_m16n8k8_tf32(float (&c)[4], const uint32_t (&a)[4],
+                                                 const uint32_t (&b)[2]) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+__device__ __forceinline__ void mma_tile_tf32x3(const float* A, int lda, const float* B, int ldb,
+                                                int ksteps, float (&c)[4], int g, int t) {
+    float c1[4] = {0.f, 0.f, 0.f, 0.f}, c2[4] = {0.f, 0.f, 0.f, 0.f};   // separate dependency chains
+#pragma unroll 4
+    for (int ks = 0; ks < ksteps; ++ks) {
+        const float* a_ = A + 8 * ks;
+        const float* b_ = B + (8 * ks) * ldb;
+        const float af[4] = {a_[g * lda + t], a_[(g + 8) * lda + t], a_[g * lda + t + 4],
+                             a_[(g + 8) * lda + t + 4]};
+        const float bf[2] = {b_[t * ldb + g], b_[(t + 4) * ldb + g]};
+        uint32_t ah[4], al[4], bh[2], bl[2];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) split_tf32(af[i], ah[i], al[i]);
+#pragma unroll
+        for (int i = 0; i < 2; ++i) split_tf32(bf[i], bh[i], bl[i]);
+        mma_m16n8k8_tf32(c1, al, bh);
+        mma_m16n8k8_tf32(c2, ah, bl);
+        mma_m16n8k8_tf32(c, ah, bh);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) c[i] += c1[i] + c2[i];
+}
+
 // T = (I + A)^{-1} for the strictly lower-triangular 64x64 A in sA (row-major, stride kLdA),
-// in place, by 256 threads: four 16x16 diagonal blocks by forward substitution, then the
+// in place, by 256 threads: four 16x16 diagonal blocks by forward substitution in fp32, then the
 // off-diagonal blocks by block elimination at block sizes 16 and 32
-//     [[Ta, 0], [X, Tb]],  X = -Tb (A_ba Ta).
-// fp32 throughout.  Ends with a __syncthreads().
+//     [[Ta, 0], [X, Tb]],  X = -Tb (A_ba Ta),
+// whose small products run on the legacy mma.sync path with split-tf32 operands (fp32-level
+// accuracy; tcgen05 needs M >= 64).  Ends with a __syncthreads().
 #ifdef GDN_PHASE_TIMING
 #define ST(k) do { if (tid == 0 && st_out) st_out[k] = clock64(); } while (0)
 #else
@@ -146,72 +186,46 @@ __device__ __forceinline__ void solve_unit_lower_64(float* sA, float* scr, int t
     ST(1);
     __syncthreads();
     ST(2);
-    // ---- 16-blocks (1,0) and (3,2): two chains of two 16x16x16 products, 128 threads each,
-    //      thread = (row ty, two columns 2tx, 2tx+1)
+    // ---- off-diagonal blocks on the tensor cores (mma.sync m16n8k8, 3xTF32: fp32-level accuracy)
+    const int warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+    // 16-blocks (1,0) and (3,2): X = A_IJ T_JJ, then T_IJ = -T_II X.  Four 16x8 tiles, warps 0-3.
     {
-        const int pr = tid >> 7, t = tid & 127, ty = t >> 3, tx = t & 7;
+        const int pr = warp >> 1, nb = warp & 1;            // pair, 8-column block
         const int I = 2 * pr + 1, J = 2 * pr;
-        float* X = scr + pr * (16 * 20);
-        float2 acc = make_float2(0.f, 0.f);
-#pragma unroll
-        for (int k0 = 0; k0 < 16; k0 += 4) {
-            const float4 a = *reinterpret_cast<const float4*>(sA + (16 * I + ty) * kLdA + 16 * J + k0);
-            const float av[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-                const float2 b = *reinterpret_cast<const float2*>(sA + (16 * J + k0 + kk) * kLdA + 16 * J + 2 * tx);
-                acc.x = fmaf(av[kk], b.x, acc.x); acc.y = fmaf(av[kk], b.y, acc.y);
-            }
+        float* X = scr + pr * (16 * 24);
+        float c[4] = {0.f, 0.f, 0.f, 0.f};
+        if (warp < 4) {
+            mma_tile_tf32x3(sA + (16 * I) * kLdA + 16 * J, kLdA, sA + (16 * J) * kLdA + 16 * J + 8 * nb,
+                            kLdA, 2, c, g, t);
+            *reinterpret_cast<float2*>(X + g * 24 + 8 * nb + 2 * t) = make_float2(c[0], c[1]);
+            *reinterpret_cast<float2*>(X + (g + 8) * 24 + 8 * nb + 2 * t) = make_float2(c[2], c[3]);
         }
-        *reinterpret_cast<float2*>(X + ty * 20 + 2 * tx) = acc;
         __syncthreads();
         ST(3);
-        acc = make_float2(0.f, 0.f);
-#pragma unroll
-        for (int k0 = 0; k0 < 16; k0 += 4) {
-            const float4 a = *reinterpret_cast<const float4*>(sA + (16 * I + ty) * kLdA + 16 * I + k0);
-            const float av[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-                const float2 b = *reinterpret_cast<const float2*>(X + (k0 + kk) * 20 + 2 * tx);
-                acc.x = fmaf(-av[kk], b.x, acc.x); acc.y = fmaf(-av[kk], b.y, acc.y);
-            }
+        if (warp < 4) {
+            c[0] = c[1] = c[2] = c[3] = 0.f;
+            mma_tile_tf32x3(sA + (16 * I) * kLdA + 16 * I, kLdA, X + 8 * nb, 24, 2, c, g, t);
+            float* dst = sA + (16 * I) * kLdA + 16 * J + 8 * nb;
+            *reinterpret_cast<float2*>(dst + g * kLdA + 2 * t) = make_float2(-c[0], -c[1]);
+            *reinterpret_cast<float2*>(dst + (g + 8) * kLdA + 2 * t) = make_float2(-c[2], -c[3]);
         }
-        *reinterpret_cast<float2*>(sA + (16 * I + ty) * kLdA + 16 * J + 2 * tx) = acc;
     }
     __syncthreads();
     ST(4);
-    // ---- 32-block (1,0): Y = A_ba Ta, then X = -Tb Y; thread = (row ty, columns 4tx..4tx+3)
+    // 32-block (1,0): Y = A_ba Ta, then X = -Tb Y.  Eight 16x8 tiles, one per warp.
     {
-        const int ty = tid >> 3, tx = tid & 7;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-        for (int k0 = 0; k0 < 32; k0 += 4) {
-            const float4 a = *reinterpret_cast<const float4*>(sA + (32 + ty) * kLdA + k0);
-            const float av[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-                const float4 b = *reinterpret_cast<const float4*>(sA + (k0 + kk) * kLdA + 4 * tx);
-                acc.x = fmaf(av[kk], b.x, acc.x); acc.y = fmaf(av[kk], b.y, acc.y);
-                acc.z = fmaf(av[kk], b.z, acc.z); acc.w = fmaf(av[kk], b.w, acc.w);
-            }
-        }
-        *reinterpret_cast<float4*>(scr + ty * 36 + 4 * tx) = acc;
+        const int mr = warp >> 2, nb = warp & 3;
+        float c[4] = {0.f, 0.f, 0.f, 0.f};
+        mma_tile_tf32x3(sA + (32 + 16 * mr) * kLdA, kLdA, sA + 8 * nb, kLdA, 4, c, g, t);
+        *reinterpret_cast<float2*>(scr + (16 * mr + g) * 40 + 8 * nb + 2 * t) = make_float2(c[0], c[1]);
+        *reinterpret_cast<float2*>(scr + (16 * mr + g + 8) * 40 + 8 * nb + 2 * t) = make_float2(c[2], c[3]);
         __syncthreads();
         ST(5);
-        acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-        for (int k0 = 0; k0 < 32; k0 += 4) {
-            const float4 a = *reinterpret_cast<const float4*>(sA + (32 + ty) * kLdA + 32 + k0);
-            const float av[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-                const float4 b = *reinterpret_cast<const float4*>(scr + (k0 + kk) * 36 + 4 * tx);
-                acc.x = fmaf(-av[kk], b.x, acc.x); acc.y = fmaf(-av[kk], b.y, acc.y);
-                acc.z = fmaf(-av[kk], b.z, acc.z); acc.w = fmaf(-av[kk], b.w, acc.w);
-            }
-        }
-        *reinterpret_cast<float4*>(sA + (32 + ty) * kLdA + 4 * tx) = acc;
+        c[0] = c[1] = c[2] = c[3] = 0.f;
+        mma_tile_tf32x3(sA + (32 + 16 * mr) * kLdA + 32, kLdA, scr + 8 * nb, 40, 4, c, g, t);
+        float* dst = sA + (32 + 16 * mr) * kLdA + 8 * nb;
+        *reinterpret_cast<float2*>(dst + g * kLdA + 2 * t) = make_float2(-c[0], -c[1]);
+        *reinterpret_cast<float2*>(dst + (g + 8) * kLdA + 2 * t) = make_float2(-c[2], -c[3]);
     }
     __syncthreads();
     ST(6);
@@ -259,8 +273,17 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
         mbar_init(&bar_mma, 1);
         abort_flag = 0;
         fence_barrier_init();
+        // the tiles first: everything below overlaps their flight
+        mbar_expect_tx(&bar_tma, 32768 + 16384);
+        tma_load_2d(smem + kI_QK, &maps.q, hqk * kD, ci.t0, &bar_tma);
+        tma_load_2d(smem + kI_QK + 8192, &maps.k, hqk * kD, ci.t0, &bar_tma);
+        tma_load_2d(smem + kI_QK + 16384, &maps.q, hqk * kD + 64, ci.t0, &bar_tma);
+        tma_load_2d(smem + kI_QK + 24576, &maps.k, hqk * kD + 64, ci.t0, &bar_tma);
+        tma_load_2d(smem + kI_V, &maps.v, hv * kD, ci.t0, &bar_tma);
+        tma_load_2d(smem + kI_V + 8192, &maps.v, hv * kD + 64, ci.t0, &bar_tma);
     }
     if (warp == 0) {
+        __syncwarp();
         tmem_alloc(&tmem_base_s, kIntraTmemCols);
         tmem_relinquish();
     }
@@ -303,15 +326,6 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
     const uint32_t tmem = tmem_base_s;
     PT(0);
 
-    if (tid == 0) {
-        mbar_expect_tx(&bar_tma, 32768 + 16384);
-        tma_load_2d(smem + kI_QK, &maps.q, hqk * kD, ci.t0, &bar_tma);
-        tma_load_2d(smem + kI_QK + 8192, &maps.k, hqk * kD, ci.t0, &bar_tma);
-        tma_load_2d(smem + kI_QK + 16384, &maps.q, hqk * kD + 64, ci.t0, &bar_tma);
-        tma_load_2d(smem + kI_QK + 24576, &maps.k, hqk * kD + 64, ci.t0, &bar_tma);
-        tma_load_2d(smem + kI_V, &maps.v, hv * kD, ci.t0, &bar_tma);
-        tma_load_2d(smem + kI_V + 8192, &maps.v, hv * kD + 64, ci.t0, &bar_tma);
-    }
     if (warp == 0 && !warp_wait(&bar_tma, 0)) abort_flag = 1;      // one warp polls, the rest block
     __syncthreads();
     if (abort_flag) {
@@ -683,11 +697,12 @@ prefill_state_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
                                make_sdesc_sw128(sRec + kRecW + off, 16, 1024), id64, ks > 0);
                     }
                     mma_commit(&bar_d1);
-#ifdef GDN_PHASE_TIMING
-                    PTI(6);
-                    mbar_wait(&bar_d1, j & 1);
-                    PTI(7);
-#endif
+                    if (j > 0 && j + 1 < nc) {
+                        // the other stage is free once chunk j-1's last product has retired (the
+                        // epilogue warps left it before they handed over this chunk's S)
+                        if (!wait_or_abort(&bar_y, (j - 1) & 1, abortp)) break;
+                        issue_loads(j + 1);
+                    }
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {       // Y = S Qg^T  (off the chain)
                         const uint32_t off = (ks >> 2) * 8192 + (ks & 3) * 32;
@@ -695,12 +710,6 @@ prefill_state_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
                                make_sdesc_sw128(sRec + kRecQg + off, 16, 1024), id64, ks > 0);
                     }
                     PTI(2);
-                    if (j > 0 && j + 1 < nc) {
-                        // the other stage is free once chunk j-1's last product has retired (the
-                        // epilogue warps left it before they handed over this chunk's S)
-                        if (!wait_or_abort(&bar_y, (j - 1) & 1, abortp)) break;
-                        issue_loads(j + 1);
-                    }
                     PTI(3);
                     if (!wait_or_abort(&bar_u, j & 1, abortp)) break;       // U operands in TMEM
                     tc_fence_after_sync();
