@@ -183,6 +183,12 @@ int gdn_prefill_static(const void* q, const void* k, const void* v,
 /* Human-readable name of a return code (static storage, never NULL). */
 const char* gdn_status_string(int code);
 
+/*
+ * The CUDA runtime's description of the error behind the calling thread's most
+ * recent GDN_ERR_CUDA return ("no error" if there was none).  Static storage.
+ */
+const char* gdn_last_cuda_error_string(void);
+
 /* Library version, major * 10000 + minor * 100 + patch. */
 int gdn_version(void);
 

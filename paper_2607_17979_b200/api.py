@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libgdn_b200.so")
 
 EXPORTS = ("gdn_decode", "gdn_prefill_workspace_bytes", "gdn_prefill", "gdn_prefill_recurrent",
            "gdn_prefill_static", "gdn_prefill_static_workspace_bytes", "gdn_status_string",
-           "gdn_version")
+           "gdn_last_cuda_error_string", "gdn_version")
 
 # kernels one call enqueues (for the benchmark's launch count)
 LAUNCHES_PER_DECODE = 1
@@ -45,13 +45,15 @@ _lib.gdn_prefill_static_workspace_bytes.restype = _Z
 _lib.gdn_prefill_static_workspace_bytes.argtypes = []
 _lib.gdn_status_string.restype = ctypes.c_char_p
 _lib.gdn_status_string.argtypes = [ctypes.c_int]
+_lib.gdn_last_cuda_error_string.restype = ctypes.c_char_p
 _lib.gdn_version.restype = ctypes.c_int
 
 
 class GdnError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
-        super().__init__(f"{where}: {status_string(code)} ({code})")
+        detail = f" [{_lib.gdn_last_cuda_error_string().decode()}]" if code == -6 else ""
+        super().__init__(f"{where}: {status_string(code)} ({code}){detail}")
 
 
 def status_string(code: int) -> str:

@@ -5,6 +5,15 @@
 
 namespace {
 
+thread_local cudaError_t g_last_cuda_error = cudaSuccess;
+
+// remember the runtime's own code behind a GDN_ERR_CUDA return
+inline int cuda_status(cudaError_t e) {
+    if (e == cudaSuccess) return GDN_OK;
+    g_last_cuda_error = e;
+    return GDN_ERR_CUDA;
+}
+
 inline bool misaligned(const void* p, size_t a) {
     return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0;
 }
@@ -58,8 +67,7 @@ int gdn_decode(const void* q, const void* k, const void* v, const float* g, cons
     p.o = static_cast<__nv_bfloat16*>(o);
     p.B = B; p.Hqk = Hqk; p.Hv = Hv; p.num_slots = num_slots; p.scale = scale;
     p.dev_status = dev_status;
-    return gdn::launch_decode(p, static_cast<cudaStream_t>(stream)) == cudaSuccess ? GDN_OK
-                                                                                   : GDN_ERR_CUDA;
+    return cuda_status(gdn::launch_decode(p, static_cast<cudaStream_t>(stream)));
 }
 
 size_t gdn_prefill_workspace_bytes(int32_t T, int32_t N, int32_t Hqk, int32_t Hv,
@@ -85,8 +93,7 @@ int gdn_prefill_recurrent(const void* q, const void* k, const void* v, const flo
     p.o = static_cast<__nv_bfloat16*>(o);
     p.T = T; p.N = N; p.Hqk = Hqk; p.Hv = Hv; p.num_slots = num_slots; p.scale = scale;
     p.dev_status = dev_status;
-    return gdn::launch_prefill_recurrent(p, static_cast<cudaStream_t>(stream)) == cudaSuccess
-               ? GDN_OK : GDN_ERR_CUDA;
+    return cuda_status(gdn::launch_prefill_recurrent(p, static_cast<cudaStream_t>(stream)));
 }
 
 int gdn_prefill(const void* q, const void* k, const void* v, const float* g, const float* beta,
@@ -116,8 +123,7 @@ int gdn_prefill(const void* q, const void* k, const void* v, const float* g, con
     p.dev_status = dev_status;
     cp.ws = static_cast<uint8_t*>(workspace);
     cp.lay = gdn::workspace_layout(T, N, Hv);
-    return gdn::launch_prefill_chunked(cp, static_cast<cudaStream_t>(stream)) == cudaSuccess
-               ? GDN_OK : GDN_ERR_CUDA;
+    return cuda_status(gdn::launch_prefill_chunked(cp, static_cast<cudaStream_t>(stream)));
 }
 
 const char* gdn_status_string(int code) {
@@ -133,6 +139,8 @@ const char* gdn_status_string(int code) {
         default: return "unknown status";
     }
 }
+
+const char* gdn_last_cuda_error_string(void) { return cudaGetErrorString(g_last_cuda_error); }
 
 int gdn_version(void) { return 100; }
 

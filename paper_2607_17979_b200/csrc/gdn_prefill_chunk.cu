@@ -3,22 +3,6 @@
 #include "gdn_prefill_chunk.cuh"
 #include "gdn_sm100.cuh"
 
-// Optional phase timing for development builds (-DGDN_PHASE_TIMING): thread 0 of one chosen CTA
-// accumulates clock64() deltas per phase and leaves them in the workspace header.
-#ifdef GDN_PHASE_TIMING
-#define PT_DECL long long pt_last = clock64(); long long pt_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
-#define PT(k) do { if (threadIdx.x == 0) { const long long t_ = clock64(); pt_acc[k] += t_ - pt_last; pt_last = t_; } } while (0)
-#define PTI(k) do { const long long t_ = clock64(); pt_acc[k] += t_ - pt_last; pt_last = t_; } while (0)
-#define PTI_FLUSH(cond, off, n) do { if (cond) for (int i_ = 0; i_ < (n); ++i_) reinterpret_cast<long long*>(ws + (off))[i_] = pt_acc[i_]; } while (0)
-#define PT_FLUSH(cond, off, n) do { if (threadIdx.x == 0 && (cond)) for (int i_ = 0; i_ < (n); ++i_) reinterpret_cast<long long*>(ws + (off))[i_] = pt_acc[i_]; } while (0)
-#else
-#define PT_DECL
-#define PT(k)
-#define PTI(k)
-#define PTI_FLUSH(cond, off, n)
-#define PT_FLUSH(cond, off, n)
-#endif
-
 namespace gdn {
 using namespace sm100;
 
@@ -159,13 +143,7 @@ __device__ __forceinline__ void mma_tile_tf32x3(const float* A, int lda, const f
 //     [[Ta, 0], [X, Tb]],  X = -Tb (A_ba Ta),
 // whose small products run on the legacy mma.sync path with split-tf32 operands (fp32-level
 // accuracy; tcgen05 needs M >= 64).  Ends with a __syncthreads().
-#ifdef GDN_PHASE_TIMING
-#define ST(k) do { if (tid == 0 && st_out) st_out[k] = clock64(); } while (0)
-#else
-#define ST(k)
-#endif
-__device__ __forceinline__ void solve_unit_lower_64(float* sA, float* scr, int tid, long long* st_out) {
-    ST(0);
+__device__ __forceinline__ void solve_unit_lower_64(float* sA, float* scr, int tid) {
     // ---- diagonal blocks: thread (I, j) computes column j of (I + A_II)^{-1}, right-looking
     if (tid < 64) {
         const int I = tid >> 4, j = tid & 15;
@@ -183,9 +161,7 @@ __device__ __forceinline__ void solve_unit_lower_64(float* sA, float* scr, int t
 #pragma unroll
         for (int r = 0; r < 16; ++r) blk[r * kLdA + j] = t[r];
     }
-    ST(1);
     __syncthreads();
-    ST(2);
     // ---- off-diagonal blocks on the tensor cores (mma.sync m16n8k8, 3xTF32: fp32-level accuracy)
     const int warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     // 16-blocks (1,0) and (3,2): X = A_IJ T_JJ, then T_IJ = -T_II X.  Four 16x8 tiles, warps 0-3.
@@ -201,7 +177,6 @@ __device__ __forceinline__ void solve_unit_lower_64(float* sA, float* scr, int t
             *reinterpret_cast<float2*>(X + (g + 8) * 24 + 8 * nb + 2 * t) = make_float2(c[2], c[3]);
         }
         __syncthreads();
-        ST(3);
         if (warp < 4) {
             c[0] = c[1] = c[2] = c[3] = 0.f;
             mma_tile_tf32x3(sA + (16 * I) * kLdA + 16 * I, kLdA, X + 8 * nb, 24, 2, c, g, t);
@@ -211,7 +186,6 @@ __device__ __forceinline__ void solve_unit_lower_64(float* sA, float* scr, int t
         }
     }
     __syncthreads();
-    ST(4);
     // 32-block (1,0): Y = A_ba Ta, then X = -Tb Y.  Eight 16x8 tiles, one per warp.
     {
         const int mr = warp >> 2, nb = warp & 3;
@@ -220,7 +194,6 @@ __device__ __forceinline__ void solve_unit_lower_64(float* sA, float* scr, int t
         *reinterpret_cast<float2*>(scr + (16 * mr + g) * 40 + 8 * nb + 2 * t) = make_float2(c[0], c[1]);
         *reinterpret_cast<float2*>(scr + (16 * mr + g + 8) * 40 + 8 * nb + 2 * t) = make_float2(c[2], c[3]);
         __syncthreads();
-        ST(5);
         c[0] = c[1] = c[2] = c[3] = 0.f;
         mma_tile_tf32x3(sA + (32 + 16 * mr) * kLdA + 32, kLdA, scr + 8 * nb, 40, 4, c, g, t);
         float* dst = sA + (32 + 16 * mr) * kLdA + 8 * nb;
@@ -228,7 +201,6 @@ __device__ __forceinline__ void solve_unit_lower_64(float* sA, float* scr, int t
         *reinterpret_cast<float2*>(dst + (g + 8) * kLdA + 2 * t) = make_float2(-c[2], -c[3]);
     }
     __syncthreads();
-    ST(6);
 }
 
 // Lane 0 polls the mbarrier (bounded), the other lanes block at the warp barrier instead of
@@ -267,7 +239,6 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
 
     const int tid = threadIdx.x, warp = tid >> 5;
     const int colhalf = warp >> 2;                   // which 32 of the 64 accumulator columns
-    PT_DECL
     if (tid == 0) {
         mbar_init(&bar_tma, 1);
         mbar_init(&bar_mma, 1);
@@ -324,7 +295,6 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = tmem_base_s;
-    PT(0);
 
     if (warp == 0 && !warp_wait(&bar_tma, 0)) abort_flag = 1;      // one warp polls, the rest block
     __syncthreads();
@@ -334,7 +304,6 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
         return;
     }
     tc_fence_after_sync();
-    PT(1);
 
     const uint32_t tG = tmem, tW = tmem + 64, tU = tmem + 128;
     const uint32_t sQK = smem_u32(smem + kI_QK);
@@ -357,7 +326,6 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
         return;
     }
     tc_fence_after_sync();
-    PT(2);
 
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
     float* sA = reinterpret_cast<float*>(smem + kI_A);
@@ -421,13 +389,8 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
         }
     }
     __syncthreads();
-    PT(3);
 
-    long long* st_out = nullptr;
-#ifdef GDN_PHASE_TIMING
-    if (false) st_out = reinterpret_cast<long long*>(ws + 192);
-#endif
-    solve_unit_lower_64(sA, reinterpret_cast<float*>(smem + kI_Scr), tid, st_out);
+    solve_unit_lower_64(sA, reinterpret_cast<float*>(smem + kI_Scr), tid);
 
     {   // T (fp32, row-major) -> bf16 B operands T diag(beta e^b), T diag(beta) (hi, lo)
 #pragma unroll
@@ -458,10 +421,8 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
             *reinterpret_cast<uint4*>(smem + kI_TuLo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
         }
     }
-    ST(7);
     fence_proxy_async_smem();
     __syncthreads();
-    PT(4);
 
     if (tid == 0) {
         // Qg and P are final: start their stores while the last products run
@@ -496,7 +457,6 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
         return;
     }
     tc_fence_after_sync();
-    PT(5);
 
     {   // thread (d, column half) holds W^T[d][32 tokens] and U~^T[d][32 tokens]
         const int d = (warp & 3) * 32 + (tid & 31);
@@ -538,8 +498,6 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
         bulk_commit();
         bulk_wait_read_all();
     }
-    PT(6);
-    PT_FLUSH(blockIdx.x == gridDim.x / 2 && blockIdx.y == gridDim.y / 2, 64, 7);
     if (warp == 0) tmem_dealloc(tmem, kIntraTmemCols);
 }
 
@@ -678,24 +636,36 @@ prefill_state_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
                 };
                 const uint32_t id64 = make_idesc_bf16(128, 64, false, false);
                 const uint32_t id128mn = make_idesc_bf16(128, 128, false, true);
+                // base descriptors of both stages, built once; the loop only adds offsets
+                const uint32_t sRec0 = smem_u32(smem + kS_Rec), sRec1 = sRec0 + kStageBytes;
+                const uint64_t dW0 = make_sdesc_sw128(sRec0 + kRecW, 16, 1024);
+                const uint64_t dQ0 = make_sdesc_sw128(sRec0 + kRecQg, 16, 1024);
+                const uint64_t dP0 = make_sdesc_sw128(sRec0 + kRecP, 16, 1024);
+                const uint64_t dK0 = make_sdesc_sw128(sRec0 + kS_K, 8192, 1024);
+                const uint64_t dW1 = make_sdesc_sw128(sRec1 + kRecW, 16, 1024);
+                const uint64_t dQ1 = make_sdesc_sw128(sRec1 + kRecQg, 16, 1024);
+                const uint64_t dP1 = make_sdesc_sw128(sRec1 + kRecP, 16, 1024);
+                const uint64_t dK1 = make_sdesc_sw128(sRec1 + kS_K, 8192, 1024);
+                const uint32_t tS = tmem + kT_S, tD1 = tmem + kT_D1, tD4 = tmem + kT_D4;
                 issue_loads(0);
                 if (nc > 1) issue_loads(1);
-                PT_DECL
                 for (int j = 0; j < nc; ++j) {
                     const int st = j & 1;
-                    const uint32_t sRec = smem_u32(smem + st * kStageBytes + kS_Rec);
-                    const uint32_t sK = smem_u32(smem + st * kStageBytes + kS_K);
+                    const uint64_t w = st ? dW1 : dW0, qg = st ? dQ1 : dQ0, pp = st ? dP1 : dP0,
+                                   kk = st ? dK1 : dK0;
+                    const uint32_t tY = tmem + kT_Y + st * 64;
                     if (!wait_or_abort(&bar_full[st], (j >> 1) & 1, abortp)) break;
-                    PTI(0);
                     if (!wait_or_abort(&bar_s, j & 1, abortp)) break;       // bf16 S of chunk j in TMEM
                     tc_fence_after_sync();
-                    PTI(1);
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {       // D1 = S W^T  (on the chain)
-                        const uint32_t off = (ks >> 2) * 8192 + (ks & 3) * 32;
-                        mma_ts(tmem + kT_D1, tmem + kT_S + ks * 8,
-                               make_sdesc_sw128(sRec + kRecW + off, 16, 1024), id64, ks > 0);
-                    }
+                    // D1 = S W^T  (on the chain); k-step ks reads 16 dk: 32 bytes inside a half
+                    mma_ts_c<false>(tD1, tS, w, id64);
+                    mma_ts_c<true>(tD1, tS + 8, sdesc_advance(w, 32), id64);
+                    mma_ts_c<true>(tD1, tS + 16, sdesc_advance(w, 64), id64);
+                    mma_ts_c<true>(tD1, tS + 24, sdesc_advance(w, 96), id64);
+                    mma_ts_c<true>(tD1, tS + 32, sdesc_advance(w, 8192), id64);
+                    mma_ts_c<true>(tD1, tS + 40, sdesc_advance(w, 8192 + 32), id64);
+                    mma_ts_c<true>(tD1, tS + 48, sdesc_advance(w, 8192 + 64), id64);
+                    mma_ts_c<true>(tD1, tS + 56, sdesc_advance(w, 8192 + 96), id64);
                     mma_commit(&bar_d1);
                     if (j > 0 && j + 1 < nc) {
                         // the other stage is free once chunk j-1's last product has retired (the
@@ -703,34 +673,34 @@ prefill_state_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
                         if (!wait_or_abort(&bar_y, (j - 1) & 1, abortp)) break;
                         issue_loads(j + 1);
                     }
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {       // Y = S Qg^T  (off the chain)
-                        const uint32_t off = (ks >> 2) * 8192 + (ks & 3) * 32;
-                        mma_ts(tmem + kT_Y + st * 64, tmem + kT_S + ks * 8,
-                               make_sdesc_sw128(sRec + kRecQg + off, 16, 1024), id64, ks > 0);
-                    }
-                    PTI(2);
-                    PTI(3);
+                    // Y = S Qg^T  (off the chain)
+                    mma_ts_c<false>(tY, tS, qg, id64);
+                    mma_ts_c<true>(tY, tS + 8, sdesc_advance(qg, 32), id64);
+                    mma_ts_c<true>(tY, tS + 16, sdesc_advance(qg, 64), id64);
+                    mma_ts_c<true>(tY, tS + 24, sdesc_advance(qg, 96), id64);
+                    mma_ts_c<true>(tY, tS + 32, sdesc_advance(qg, 8192), id64);
+                    mma_ts_c<true>(tY, tS + 40, sdesc_advance(qg, 8192 + 32), id64);
+                    mma_ts_c<true>(tY, tS + 48, sdesc_advance(qg, 8192 + 64), id64);
+                    mma_ts_c<true>(tY, tS + 56, sdesc_advance(qg, 8192 + 96), id64);
                     if (!wait_or_abort(&bar_u, j & 1, abortp)) break;       // U operands in TMEM
                     tc_fence_after_sync();
-                    PTI(4);
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)          // D4 = (U decayed) K   (K tile MN-major)
-                        mma_ts(tmem + kT_D4, tmem + kT_Us + ks * 8,
-                               make_sdesc_sw128(sK + ks * 2048, 8192, 1024), id128mn, ks > 0);
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        mma_ts(tmem + kT_D4, tmem + kT_UsLo + ks * 8,
-                               make_sdesc_sw128(sK + ks * 2048, 8192, 1024), id128mn, true);
+                    // D4 = (U decayed, hi + lo) K   (K tile MN-major: 16 tokens = 2048 bytes)
+                    mma_ts_c<false>(tD4, tmem + kT_Us, kk, id128mn);
+                    mma_ts_c<true>(tD4, tmem + kT_Us + 8, sdesc_advance(kk, 2048), id128mn);
+                    mma_ts_c<true>(tD4, tmem + kT_Us + 16, sdesc_advance(kk, 4096), id128mn);
+                    mma_ts_c<true>(tD4, tmem + kT_Us + 24, sdesc_advance(kk, 6144), id128mn);
+                    mma_ts_c<true>(tD4, tmem + kT_UsLo, kk, id128mn);
+                    mma_ts_c<true>(tD4, tmem + kT_UsLo + 8, sdesc_advance(kk, 2048), id128mn);
+                    mma_ts_c<true>(tD4, tmem + kT_UsLo + 16, sdesc_advance(kk, 4096), id128mn);
+                    mma_ts_c<true>(tD4, tmem + kT_UsLo + 24, sdesc_advance(kk, 6144), id128mn);
                     mma_commit(&bar_d4);
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)          // Y += U P^T
-                        mma_ts(tmem + kT_Y + st * 64, tmem + kT_U + ks * 8,
-                               make_sdesc_sw128(sRec + kRecP + ks * 32, 16, 1024), id64, true);
+                    // Y += U P^T
+                    mma_ts_c<true>(tY, tmem + kT_U, pp, id64);
+                    mma_ts_c<true>(tY, tmem + kT_U + 8, sdesc_advance(pp, 32), id64);
+                    mma_ts_c<true>(tY, tmem + kT_U + 16, sdesc_advance(pp, 64), id64);
+                    mma_ts_c<true>(tY, tmem + kT_U + 24, sdesc_advance(pp, 96), id64);
                     mma_commit(&bar_y);
-                    PTI(5);
                 }
-                PTI_FLUSH(blockIdx.x == gridDim.x - 1, 192, 8);
             }
             __syncwarp();
         } else {
@@ -750,9 +720,11 @@ prefill_state_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
                     tmem_st16(tmem + kT_S + lane_base + half * 32 + (c0 >> 1), pk);
                 }
             };
-            // o rows of chunk j from Y[j & 1]: scale, round to bf16, transpose through shared
-            // memory, write 16-byte pieces of whole rows
-            auto write_outputs = [&](int j) {
+            // o rows of chunk j from Y[j & 1], in two parts that fit the two waits of the chain:
+            // (A) scale, round to bf16, transpose into shared memory; (B) write whole rows in
+            // 16-byte pieces.  A group barrier precedes each part (all of B(j-1) before A(j),
+            // all of A(j) before B(j)).
+            auto outputs_stage = [&](int j) {
                 const uint32_t tY = tmem + kT_Y + (j & 1) * 64;
                 __nv_bfloat16* sO = reinterpret_cast<__nv_bfloat16*>(smem + kS_Out);
                 uint32_t x[16], y[16];
@@ -764,7 +736,9 @@ prefill_state_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
                     sO[(half * 32 + jj) * kD + dv] = __float2bfloat16(p.scale * __uint_as_float(x[jj]));
                     sO[(half * 32 + 16 + jj) * kD + dv] = __float2bfloat16(p.scale * __uint_as_float(y[jj]));
                 }
-                epi_group_sync();
+            };
+            auto outputs_flush = [&](int j) {
+                const __nv_bfloat16* sO = reinterpret_cast<const __nv_bfloat16*>(smem + kS_Out);
                 const int len = min(kChunk, seq_len - j * kChunk);
                 __nv_bfloat16* og = p.o + (static_cast<size_t>(seq_t0 + j * kChunk) * p.Hv + hv) * kD;
                 const size_t tok_stride = static_cast<size_t>(p.Hv) * kD;
@@ -779,16 +753,19 @@ prefill_state_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
 
             store_state_bf16();
             hand_over(&bar_s);
-            PT_DECL
             bool ok = true;
             for (int j = 0; j < nc; ++j) {
                 const int st = j & 1;
                 const uint8_t* base = smem + st * kStageBytes;
-                PT(0);
+                if (j > 0) {     // part A of the previous chunk's outputs, while D1 is in flight
+                    if (!warp_wait_or_abort(&bar_y, (j - 1) & 1, abortp)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    epi_group_sync();
+                    outputs_stage(j - 1);
+                }
                 if (!warp_wait_or_abort(&bar_full[st], (j >> 1) & 1, abortp)) { ok = false; break; }
                 if (!warp_wait_or_abort(&bar_d1, j & 1, abortp)) { ok = false; break; }
                 tc_fence_after_sync();
-                PT(1);
 
                 const float* sdec = reinterpret_cast<const float*>(base + kS_Rec + kRecDecay);
                 {   // U^T[dv][c] = U~^T - D1 for the thread's 32 tokens [32*half, 32*half+32)
@@ -832,18 +809,13 @@ prefill_state_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
                     u_block(xb, half * 32 + 16);
                 }
                 hand_over(&bar_u);
-                PT(2);
-                if (j > 0) {
-                    // the previous chunk's output rows, while this chunk's state product runs
-                    if (!warp_wait_or_abort(&bar_y, (j - 1) & 1, abortp)) { ok = false; break; }
-                    tc_fence_after_sync();
-                    write_outputs(j - 1);
+                if (j > 0) {     // part B, while this chunk's state product is in flight
+                    epi_group_sync();
+                    outputs_flush(j - 1);
                 }
-                PT(5);
 
                 if (!warp_wait_or_abort(&bar_d4, j & 1, abortp)) { ok = false; break; }
                 tc_fence_after_sync();
-                PT(3);
                 {   // S <- e^{b_C} S + D4 on the thread's 64 dk columns; refresh the bf16 copy
                     const float gC = reinterpret_cast<const float*>(base + kS_Rec + kRecGammaC)[0];
 #pragma unroll
@@ -861,18 +833,16 @@ prefill_state_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
                     store_state_bf16();
                 }
                 hand_over(&bar_s);
-                PT(4);
             }
             if (ok) {
                 if (warp_wait_or_abort(&bar_y, (nc - 1) & 1, abortp)) {
                     tc_fence_after_sync();
-                    // inside the loop the next chunk's barriers keep a fast warp from refilling
-                    // the staging tile while a slow one still reads it; here nothing else does
                     epi_group_sync();
-                    write_outputs(nc - 1);
+                    outputs_stage(nc - 1);
+                    epi_group_sync();
+                    outputs_flush(nc - 1);
                 }
             }
-            PT_FLUSH(blockIdx.x == gridDim.x - 1, 128, 6);
         }
         tc_fence_before_sync();
         __syncthreads();
