@@ -131,6 +131,23 @@ int gdn_prefill(const void* q, const void* k, const void* v,
                 int32_t* dev_status, void* stream);
 
 /*
+ * gdn_prefill routes by the longest sequence: at most GDN_RECURRENT_MAX_SEQLEN
+ * tokens (by max_seqlen_hint if given, else by the bound T) goes to the
+ * token-by-token kernel, anything longer to the chunked kernels.  The two
+ * routes below can also be called directly; arguments are gdn_prefill's.
+ */
+#define GDN_RECURRENT_MAX_SEQLEN 16
+int gdn_prefill_chunked(const void* q, const void* k, const void* v,
+                        const float* g, const float* beta, const int32_t* cu_seqlens,
+                        const float* init_state, float* final_state, const int32_t* slot_idx,
+                        void* o,
+                        int32_t T, int32_t N, int32_t max_seqlen_hint,
+                        int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv, int32_t chunk,
+                        int32_t num_slots, float scale,
+                        void* workspace, size_t workspace_bytes,
+                        int32_t* dev_status, void* stream);
+
+/*
  * gdn_prefill_recurrent - the same operator and arguments as gdn_prefill,
  * evaluated token by token on the CUDA cores (no chunking, no workspace).  The
  * rows of a state tile evolve independently under the gated delta rule, so the

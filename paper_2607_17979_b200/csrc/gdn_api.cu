@@ -96,12 +96,12 @@ int gdn_prefill_recurrent(const void* q, const void* k, const void* v, const flo
     return cuda_status(gdn::launch_prefill_recurrent(p, static_cast<cudaStream_t>(stream)));
 }
 
-int gdn_prefill(const void* q, const void* k, const void* v, const float* g, const float* beta,
-                const int32_t* cu_seqlens, const float* init_state, float* final_state,
-                const int32_t* slot_idx, void* o, int32_t T, int32_t N, int32_t max_seqlen_hint,
-                int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv, int32_t chunk,
-                int32_t num_slots, float scale, void* workspace, size_t workspace_bytes,
-                int32_t* dev_status, void* stream) {
+int gdn_prefill_chunked(const void* q, const void* k, const void* v, const float* g,
+                        const float* beta, const int32_t* cu_seqlens, const float* init_state,
+                        float* final_state, const int32_t* slot_idx, void* o, int32_t T, int32_t N,
+                        int32_t max_seqlen_hint, int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv,
+                        int32_t chunk, int32_t num_slots, float scale, void* workspace,
+                        size_t workspace_bytes, int32_t* dev_status, void* stream) {
     (void)max_seqlen_hint;
     if (chunk != gdn::kChunk) return GDN_ERR_SHAPE;
     const int rc = check_prefill(q, k, v, g, beta, cu_seqlens, init_state, final_state, o,
@@ -124,6 +124,37 @@ int gdn_prefill(const void* q, const void* k, const void* v, const float* g, con
     cp.ws = static_cast<uint8_t*>(workspace);
     cp.lay = gdn::workspace_layout(T, N, Hv);
     return cuda_status(gdn::launch_prefill_chunked(cp, static_cast<cudaStream_t>(stream)));
+}
+
+int gdn_prefill(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                const int32_t* cu_seqlens, const float* init_state, float* final_state,
+                const int32_t* slot_idx, void* o, int32_t T, int32_t N, int32_t max_seqlen_hint,
+                int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv, int32_t chunk,
+                int32_t num_slots, float scale, void* workspace, size_t workspace_bytes,
+                int32_t* dev_status, void* stream) {
+    // Route: a batch whose longest sequence is at most GDN_RECURRENT_MAX_SEQLEN tokens goes to the
+    // token-by-token kernel (one launch, no workspace traffic); everything else is chunked.  The
+    // length is known on the host only through the caller's hint or the bound T.
+    const int32_t longest = (max_seqlen_hint > 0 && max_seqlen_hint < T) ? max_seqlen_hint : T;
+    if (chunk == gdn::kChunk && T > 0 && N > 0 && longest <= GDN_RECURRENT_MAX_SEQLEN) {
+        // same validation of the workspace arguments as the chunked route, so that a call does
+        // not start failing when its batch grows
+        if (!workspace) {
+            const int rc = check_prefill(q, k, v, g, beta, cu_seqlens, init_state, final_state, o,
+                                         T, N, Hqk, Hv, dk, dv, num_slots);
+            return rc != GDN_OK ? rc : GDN_ERR_NULL;
+        }
+        if (misaligned(workspace, 256)) return GDN_ERR_ALIGN;
+        if (workspace_bytes < gdn_prefill_workspace_bytes(T, N, Hqk, Hv, dk, dv, chunk))
+            return check_heads(Hqk, Hv, dk, dv) != GDN_OK ? check_heads(Hqk, Hv, dk, dv)
+                                                          : GDN_ERR_WORKSPACE;
+        return gdn_prefill_recurrent(q, k, v, g, beta, cu_seqlens, init_state, final_state,
+                                     slot_idx, o, T, N, Hqk, Hv, dk, dv, num_slots, scale,
+                                     dev_status, stream);
+    }
+    return gdn_prefill_chunked(q, k, v, g, beta, cu_seqlens, init_state, final_state, slot_idx, o,
+                               T, N, max_seqlen_hint, Hqk, Hv, dk, dv, chunk, num_slots, scale,
+                               workspace, workspace_bytes, dev_status, stream);
 }
 
 const char* gdn_status_string(int code) {

@@ -28,9 +28,14 @@ __device__ __forceinline__ void st_stream(float4* p, const float4& r) {
                  :: "l"(p), "f"(r.x), "f"(r.y), "f"(r.z), "f"(r.w) : "memory");
 }
 
+// kPasses = 4: one CTA per tile (16 rows per warp).  kPasses = 1: a tile is split over four CTAs
+// of 32 rows each (rows evolve independently), used when there are too few tiles to fill the GPU.
+template <int kPasses>
 __global__ void __launch_bounds__(kDecodeThreads, 2)
 decode_kernel(const DecodeParams p) {
-    const int unit = blockIdx.x;
+    constexpr int kSplit = 4 / kPasses;
+    const int unit = blockIdx.x / kSplit;
+    const int part = blockIdx.x - unit * kSplit;
     const int i = unit / p.Hv;
     const int hv = unit - i * p.Hv;
     const int hqk = hv / (p.Hv / p.Hqk);
@@ -42,16 +47,16 @@ decode_kernel(const DecodeParams p) {
     __nv_bfloat16* o_row = p.o + (static_cast<size_t>(i) * p.Hv + hv) * kD;
     const int slot = p.slot_idx ? p.slot_idx[i] : i;
     if (slot < 0 || slot >= p.num_slots) {
-        if (slot >= p.num_slots && threadIdx.x == 0) report(p.dev_status, kDevBadSlot);
-        if (threadIdx.x < kD) o_row[threadIdx.x] = __float2bfloat16(0.f);
+        if (slot >= p.num_slots && threadIdx.x == 0 && part == 0) report(p.dev_status, kDevBadSlot);
+        if (threadIdx.x < kD / kSplit) o_row[part * (kD / kSplit) + threadIdx.x] = __float2bfloat16(0.f);
         return;
     }
 
     float* tile = p.pool + (static_cast<size_t>(slot) * p.Hv + hv) * (kD * kD);
-    const int row0 = warp * 16 + rsel;
-    float4 s[4][4];
+    const int row0 = part * (kD / kSplit) + warp * (4 * kPasses) + rsel;
+    float4 s[kPasses][4];
 #pragma unroll
-    for (int ps = 0; ps < 4; ++ps)
+    for (int ps = 0; ps < kPasses; ++ps)
 #pragma unroll
         for (int j = 0; j < 4; ++j)
             s[ps][j] = ld_stream(reinterpret_cast<const float4*>(
@@ -71,12 +76,12 @@ decode_kernel(const DecodeParams p) {
     kq = sum8(kq);
     const float alpha = expf(p.g[static_cast<size_t>(i) * p.Hv + hv]);
     const float beta = p.beta[static_cast<size_t>(i) * p.Hv + hv];
-    float vj[4];
+    float vj[kPasses];
 #pragma unroll
-    for (int ps = 0; ps < 4; ++ps) vj[ps] = __bfloat162float(vp[row0 + ps * 4]);
+    for (int ps = 0; ps < kPasses; ++ps) vj[ps] = __bfloat162float(vp[row0 + ps * 4]);
 
 #pragma unroll
-    for (int ps = 0; ps < 4; ++ps) {
+    for (int ps = 0; ps < kPasses; ++ps) {
         float pk = 0.f, pq = 0.f;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -103,7 +108,15 @@ decode_kernel(const DecodeParams p) {
 cudaError_t launch_decode(const DecodeParams& p, cudaStream_t stream) {
     const long long units = static_cast<long long>(p.B) * p.Hv;
     if (units == 0) return cudaSuccess;
-    decode_kernel<<<static_cast<unsigned>(units), kDecodeThreads, 0, stream>>>(p);
+    // below about two CTAs per SM of whole tiles, quarter tiles spread the same bytes over four
+    // times as many SMs (the state rows are independent)
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess)
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (units < 2LL * sms)
+        decode_kernel<1><<<static_cast<unsigned>(units * 4), kDecodeThreads, 0, stream>>>(p);
+    else
+        decode_kernel<4><<<static_cast<unsigned>(units), kDecodeThreads, 0, stream>>>(p);
     return cudaGetLastError();
 }
 

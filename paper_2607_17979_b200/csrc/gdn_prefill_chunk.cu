@@ -74,19 +74,24 @@ prefill_prep_kernel(const int32_t* __restrict__ cu, int32_t T, int32_t N, uint8_
 // K1: intra-chunk quantities, one CTA (256 threads) per (chunk, v-head).
 // =============================================================================================
 constexpr int kIntraThreads = 256;
-constexpr uint32_t kIntraTmemCols = 256;
+constexpr uint32_t kIntraTmemCols = 128;
 constexpr int kLdA = 68;               // row stride (floats) of the fp32 A / T matrix
-// shared memory map (bytes from a 1024-aligned base)
+// Shared memory map (bytes from a 1024-aligned base).  Regions are reused as their contents die
+// so that three CTAs fit on an SM:
+//   R1  Q/K tiles.  Q halves -> Qg image (stored early) -> T_w and T_u(hi);  K halves -> W image.
+//   R2  A, then T, in fp32 plus the solve scratch -> V tile (loaded after the solve).
+//   R3  P image (stored early) -> T_u(lo).
 constexpr uint32_t kI_QK = 0;          // 2 halves x [128 rows x 128 B]: rows 0-63 Q, 64-127 K
-constexpr uint32_t kI_V = 32768;       // 2 halves x [64 x 128 B]
-constexpr uint32_t kI_Tw = 49152;      // T diag(beta e^b)  [64 r x 64 i] bf16, K-major SW128
-constexpr uint32_t kI_Tu = 57344;      // T diag(beta) rounded to bf16 ...
-constexpr uint32_t kI_TuLo = 65536;    // ... and the bf16 remainder (hi + lo carries ~16 bits)
-constexpr uint32_t kI_P = 73728;       // P image staging
-constexpr uint32_t kI_A = 81920;       // A, then T in place: fp32 [64][kLdA]
+constexpr uint32_t kI_Tw = 0;          // over Q half 0: T diag(beta e^b) [64 r x 64 i] bf16, K-major
+constexpr uint32_t kI_Tu = 16384;      // over Q half 1: T diag(beta) rounded to bf16 ...
+constexpr uint32_t kI_A = 32768;       // A, then T in place: fp32 [64][kLdA]
 constexpr uint32_t kI_Scr = kI_A + 64 * kLdA * 4;      // solve scratch, fp32 [32][40]
-constexpr uint32_t kI_End = kI_Scr + 32 * 40 * 4;
+constexpr uint32_t kI_V = 32768;       // over A: 2 halves x [64 x 128 B]
+constexpr uint32_t kI_P = 32768 + 22528;               // P image staging
+constexpr uint32_t kI_TuLo = kI_P;     // ... and the bf16 remainder of T diag(beta)
+constexpr uint32_t kI_End = kI_P + 8192;
 constexpr uint32_t kIntraSmem = kI_End + 1024;         // + alignment slack
+static_assert(kI_Scr + 32 * 40 * 4 <= kI_P, "solve scratch overlaps the P image");
 
 struct TensorMaps {
     CUtensorMap q, k, v;
@@ -215,7 +220,7 @@ __device__ __forceinline__ uint32_t scale_bf16x2(uint32_t packed, float f) {
     return pack_bf16(__uint_as_float(packed << 16) * f, __uint_as_float(packed & 0xffff0000u) * f);
 }
 
-__global__ void __launch_bounds__(kIntraThreads, 2)
+__global__ void __launch_bounds__(kIntraThreads, 3)
 prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParams p, uint8_t* ws,
                      const WorkspaceLayout lay) {
     const int c = blockIdx.x;
@@ -229,7 +234,7 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                                ~static_cast<uintptr_t>(1023));
-    __shared__ uint64_t bar_tma, bar_mma;
+    __shared__ uint64_t bar_tma, bar_v, bar_mma;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_flag;
     __shared__ __align__(16) float s_b2[kChunk];     // b_r log2(e): inclusive log-decay prefix
@@ -241,17 +246,16 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
     const int colhalf = warp >> 2;                   // which 32 of the 64 accumulator columns
     if (tid == 0) {
         mbar_init(&bar_tma, 1);
+        mbar_init(&bar_v, 1);
         mbar_init(&bar_mma, 1);
         abort_flag = 0;
         fence_barrier_init();
-        // the tiles first: everything below overlaps their flight
-        mbar_expect_tx(&bar_tma, 32768 + 16384);
+        // Q and K first: everything below overlaps their flight (V comes later, over dead data)
+        mbar_expect_tx(&bar_tma, 32768);
         tma_load_2d(smem + kI_QK, &maps.q, hqk * kD, ci.t0, &bar_tma);
         tma_load_2d(smem + kI_QK + 8192, &maps.k, hqk * kD, ci.t0, &bar_tma);
         tma_load_2d(smem + kI_QK + 16384, &maps.q, hqk * kD + 64, ci.t0, &bar_tma);
         tma_load_2d(smem + kI_QK + 24576, &maps.k, hqk * kD + 64, ci.t0, &bar_tma);
-        tma_load_2d(smem + kI_V, &maps.v, hv * kD, ci.t0, &bar_tma);
-        tma_load_2d(smem + kI_V + 8192, &maps.v, hv * kD + 64, ci.t0, &bar_tma);
     }
     if (warp == 0) {
         __syncwarp();
@@ -295,17 +299,21 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = tmem_base_s;
+    // On a timeout: flag it, let thread 0 drain what it has in flight, free TMEM, leave.
+    auto bail = [&](bool stores_pending) {
+        if (tid == 0) {
+            report(p.dev_status, kDevTimeout);
+            if (stores_pending) bulk_wait_read_all();
+        }
+        if (warp == 0) tmem_dealloc(tmem, kIntraTmemCols);
+    };
 
     if (warp == 0 && !warp_wait(&bar_tma, 0)) abort_flag = 1;      // one warp polls, the rest block
     __syncthreads();
-    if (abort_flag) {
-        if (tid == 0) report(p.dev_status, kDevTimeout);
-        if (warp == 0) tmem_dealloc(tmem, kIntraTmemCols);
-        return;
-    }
+    if (abort_flag) { bail(false); return; }
     tc_fence_after_sync();
 
-    const uint32_t tG = tmem, tW = tmem + 64, tU = tmem + 128;
+    const uint32_t tG = tmem, tW = tmem, tU = tmem + 64;     // W reuses the Gram columns
     const uint32_t sQK = smem_u32(smem + kI_QK);
     if (tid == 0) {
         // [Q;K] (128 x 128, K-major) times K^T: lanes 0-63 = q.k, lanes 64-127 = k.k
@@ -318,60 +326,58 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
         }
         mma_commit(&bar_mma);
     }
-    if (warp == 0 && !warp_wait(&bar_mma, 0)) abort_flag = 1;      // one warp polls, the rest block
+    if (warp == 0 && !warp_wait(&bar_mma, 0)) abort_flag = 1;
     __syncthreads();
-    if (abort_flag) {
-        if (tid == 0) report(p.dev_status, kDevTimeout);
-        if (warp == 0) tmem_dealloc(tmem, kIntraTmemCols);
-        return;
-    }
+    if (abort_flag) { bail(false); return; }
     tc_fence_after_sync();
 
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
     float* sA = reinterpret_cast<float*>(smem + kI_A);
     {
         // Accumulator row of this thread: TMEM lane 32 (warp % 4) + lane; lanes 0-63 hold q.k
-        // rows (-> P), lanes 64-127 hold k.k rows (-> A).  The thread covers 32 of the 64 columns.
+        // rows (-> P), lanes 64-127 hold k.k rows (-> A).  The thread covers 32 of the 64 columns,
+        // 16 at a time.
         const int row = (warp & 3) * 32 + (tid & 31);
         const int r = row & 63;
         const bool is_p = row < 64;
-        const int cbase = colhalf * 32;
         const float br2 = s_b2[r];
         const float rowscale = is_p ? 1.f : s_beta[r];
         const int limit = is_p ? r : r - 1;              // keep columns i <= limit
-        uint32_t xa[16], xb[16];
-        tmem_ld16(tG + lane_base + cbase, xa);
-        tmem_ld16(tG + lane_base + cbase + 16, xb);
-        tmem_wait_ld();
-        float val[32];
 #pragma unroll
-        for (int q4 = 0; q4 < 8; ++q4) {
-            const float4 bb = *reinterpret_cast<const float4*>(s_b2 + cbase + 4 * q4);
-            const float bv[4] = {bb.x, bb.y, bb.z, bb.w};
+        for (int step = 0; step < 2; ++step) {
+            const int cbase = colhalf * 32 + step * 16;
+            uint32_t x[16];
+            tmem_ld16(tG + lane_base + cbase, x);
+            tmem_wait_ld();
+            float val[16];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int jj = 4 * q4 + e;
-                const float x = __uint_as_float(jj < 16 ? xa[jj] : xb[jj - 16]);
-                const bool keep = cbase + jj <= limit;
-                const float dec = ex2_approx(keep ? br2 - bv[e] : 0.f);   // e^{b_r - b_i}
-                val[jj] = keep ? rowscale * dec * x : 0.f;
+            for (int q4 = 0; q4 < 4; ++q4) {
+                const float4 bb = *reinterpret_cast<const float4*>(s_b2 + cbase + 4 * q4);
+                const float bv[4] = {bb.x, bb.y, bb.z, bb.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int jj = 4 * q4 + e;
+                    const bool keep = cbase + jj <= limit;
+                    const float dec = ex2_approx(keep ? br2 - bv[e] : 0.f);   // e^{b_r - b_i}
+                    val[jj] = keep ? rowscale * dec * __uint_as_float(x[jj]) : 0.f;
+                }
             }
-        }
-        if (is_p) {
+            if (is_p) {
 #pragma unroll
-            for (int h = 0; h < 4; ++h) {
-                uint4 w;
-                w.x = pack_bf16(val[8 * h + 0], val[8 * h + 1]);
-                w.y = pack_bf16(val[8 * h + 2], val[8 * h + 3]);
-                w.z = pack_bf16(val[8 * h + 4], val[8 * h + 5]);
-                w.w = pack_bf16(val[8 * h + 6], val[8 * h + 7]);
-                *reinterpret_cast<uint4*>(smem + kI_P + sw128_offset(r, (cbase >> 3) + h)) = w;
+                for (int h = 0; h < 2; ++h) {
+                    uint4 w;
+                    w.x = pack_bf16(val[8 * h + 0], val[8 * h + 1]);
+                    w.y = pack_bf16(val[8 * h + 2], val[8 * h + 3]);
+                    w.z = pack_bf16(val[8 * h + 4], val[8 * h + 5]);
+                    w.w = pack_bf16(val[8 * h + 6], val[8 * h + 7]);
+                    *reinterpret_cast<uint4*>(smem + kI_P + sw128_offset(r, (cbase >> 3) + h)) = w;
+                }
+            } else {
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4)
+                    *reinterpret_cast<float4*>(sA + r * kLdA + cbase + 4 * q4) =
+                        make_float4(val[4 * q4], val[4 * q4 + 1], val[4 * q4 + 2], val[4 * q4 + 3]);
             }
-        } else {
-#pragma unroll
-            for (int q4 = 0; q4 < 8; ++q4)
-                *reinterpret_cast<float4*>(sA + r * kLdA + cbase + 4 * q4) =
-                    make_float4(val[4 * q4], val[4 * q4 + 1], val[4 * q4 + 2], val[4 * q4 + 3]);
         }
     }
     {   // Q rows scaled by e^{b_r}, in place (the Gram product has consumed Q): this is the Qg image
@@ -388,9 +394,21 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
             *ptr = w;
         }
     }
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
     __syncthreads();
+    if (tid == 0) {
+        // Qg and P are final: store them now; their shared memory is reused after the solve
+        bulk_store(rec + kRecQg, smem + kI_QK, 8192);
+        bulk_store(rec + kRecQg + 8192, smem + kI_QK + 16384, 8192);
+        bulk_store(rec + kRecP, smem + kI_P, 8192);
+        bulk_commit();
+    }
 
     solve_unit_lower_64(sA, reinterpret_cast<float*>(smem + kI_Scr), tid);
+
+    if (tid == 0) bulk_wait_read_all();      // the Q halves and the P image have been read out
+    __syncthreads();
 
     {   // T (fp32, row-major) -> bf16 B operands T diag(beta e^b), T diag(beta) (hi, lo)
 #pragma unroll
@@ -424,21 +442,56 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
     fence_proxy_async_smem();
     __syncthreads();
 
+    const uint32_t sV = smem_u32(smem + kI_V);
     if (tid == 0) {
-        // Qg and P are final: start their stores while the last products run
-        bulk_store(rec + kRecQg, smem + kI_QK, 8192);
-        bulk_store(rec + kRecQg + 8192, smem + kI_QK + 16384, 8192);
-        bulk_store(rec + kRecP, smem + kI_P, 8192);
-        bulk_commit();
-        // W^T (dk x r) = K^T (MN-major A from the K tile) times T_w^T ; U~^T (dv x r) likewise from V
+        // V into the space the solve has left; meanwhile W^T (dk x r) = K^T T_w^T with the raw K
+        // tile read MN-major
+        mbar_expect_tx(&bar_v, 16384);
+        tma_load_2d(smem + kI_V, &maps.v, hv * kD, ci.t0, &bar_v);
+        tma_load_2d(smem + kI_V + 8192, &maps.v, hv * kD + 64, ci.t0, &bar_v);
         const uint32_t idesc = make_idesc_bf16(128, 64, true, false);
-        const uint32_t sTw = smem_u32(smem + kI_Tw), sTu = smem_u32(smem + kI_Tu);
-        const uint32_t sTuLo = smem_u32(smem + kI_TuLo);
-        const uint32_t sV = smem_u32(smem + kI_V);
+        const uint32_t sTw = smem_u32(smem + kI_Tw);
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks)
             mma_ss(tW, make_sdesc_sw128(sQK + 8192 + ks * 2048, 16384, 1024),
                    make_sdesc_sw128(sTw + ks * 32, 16, 1024), idesc, ks > 0);
+        mma_commit(&bar_mma);
+    }
+    if (warp == 0 && !warp_wait(&bar_mma, 1)) abort_flag = 1;
+    __syncthreads();
+    if (abort_flag) { bail(false); return; }      // nothing of thread 0's stores is pending here
+    tc_fence_after_sync();
+
+    const int d = (warp & 3) * 32 + (tid & 31);   // TMEM lane of this thread: a dk / dv index
+    {   // W^T[d][32 tokens] -> bf16 -> W image staged over the (now dead) K halves
+        uint8_t* sW = smem + kI_QK + 8192 + (d >> 6) * 16384;
+        const uint32_t wcol = ((d & 7) << 1);
+        const uint32_t wchunk = (d & 63) >> 3;
+#pragma unroll
+        for (int step = 0; step < 2; ++step) {
+            const int cbase = colhalf * 32 + step * 16;
+            uint32_t x[16];
+            tmem_ld16(tW + lane_base + cbase, x);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                *reinterpret_cast<__nv_bfloat16*>(sW + sw128_offset(cbase + j, wchunk) + wcol) =
+                    __float2bfloat16(__uint_as_float(x[j]));
+        }
+    }
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    if (warp == 0 && !warp_wait(&bar_v, 0)) abort_flag = 1;        // V has landed
+    __syncthreads();
+    if (abort_flag) { bail(false); return; }
+    tc_fence_after_sync();
+    if (tid == 0) {
+        bulk_store(rec + kRecW, smem + kI_QK + 8192, 8192);
+        bulk_store(rec + kRecW + 8192, smem + kI_QK + 24576, 8192);
+        bulk_commit();
+        // U~^T (dv x r) = V^T T_u^T with T_u = hi + lo
+        const uint32_t idesc = make_idesc_bf16(128, 64, true, false);
+        const uint32_t sTu = smem_u32(smem + kI_Tu), sTuLo = smem_u32(smem + kI_TuLo);
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks)
             mma_ss(tU, make_sdesc_sw128(sV + ks * 2048, 8192, 1024),
@@ -449,55 +502,29 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
                    make_sdesc_sw128(sTuLo + ks * 32, 16, 1024), idesc, true);
         mma_commit(&bar_mma);
     }
-    if (warp == 0 && !warp_wait(&bar_mma, 1)) abort_flag = 1;      // one warp polls, the rest block
+    if (warp == 0 && !warp_wait(&bar_mma, 0)) abort_flag = 1;
     __syncthreads();
-    if (abort_flag) {
-        if (tid == 0) { report(p.dev_status, kDevTimeout); bulk_wait_read_all(); }
-        if (warp == 0) tmem_dealloc(tmem, kIntraTmemCols);
-        return;
-    }
+    if (abort_flag) { bail(true); return; }
     tc_fence_after_sync();
 
-    {   // thread (d, column half) holds W^T[d][32 tokens] and U~^T[d][32 tokens]
-        const int d = (warp & 3) * 32 + (tid & 31);
-        const int cbase = colhalf * 32;
-        // the K tile is dead now: stage W half (d / 64) over K's half (d / 64)
-        uint8_t* sW = smem + kI_QK + 8192 + (d >> 6) * 16384;
-        const uint32_t wcol = ((d & 7) << 1);
-        const uint32_t wchunk = (d & 63) >> 3;
+    {   // U~^T[d][32 tokens] -> record, [token group][dv][4 tokens] fp32
         float4* urec = reinterpret_cast<float4*>(rec + kRecU);
-        uint32_t xa[16], xb[16], ya[16], yb[16];
-        tmem_ld16(tW + lane_base + cbase, xa);
-        tmem_ld16(tW + lane_base + cbase + 16, xb);
-        tmem_ld16(tU + lane_base + cbase, ya);
-        tmem_ld16(tU + lane_base + cbase + 16, yb);
-        tmem_wait_ld();
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            *reinterpret_cast<__nv_bfloat16*>(sW + sw128_offset(cbase + j, wchunk) + wcol) =
-                __float2bfloat16(__uint_as_float(xa[j]));
-            *reinterpret_cast<__nv_bfloat16*>(sW + sw128_offset(cbase + 16 + j, wchunk) + wcol) =
-                __float2bfloat16(__uint_as_float(xb[j]));
-        }
+        for (int step = 0; step < 2; ++step) {
+            const int cbase = colhalf * 32 + step * 16;
+            uint32_t y[16];
+            tmem_ld16(tU + lane_base + cbase, y);
+            tmem_wait_ld();
 #pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {
-            urec[((cbase >> 2) + q4) * kD + d] =
-                make_float4(__uint_as_float(ya[4 * q4]), __uint_as_float(ya[4 * q4 + 1]),
-                            __uint_as_float(ya[4 * q4 + 2]), __uint_as_float(ya[4 * q4 + 3]));
-            urec[((cbase >> 2) + 4 + q4) * kD + d] =
-                make_float4(__uint_as_float(yb[4 * q4]), __uint_as_float(yb[4 * q4 + 1]),
-                            __uint_as_float(yb[4 * q4 + 2]), __uint_as_float(yb[4 * q4 + 3]));
+            for (int q4 = 0; q4 < 4; ++q4)
+                urec[((cbase >> 2) + q4) * kD + d] =
+                    make_float4(__uint_as_float(y[4 * q4]), __uint_as_float(y[4 * q4 + 1]),
+                                __uint_as_float(y[4 * q4 + 2]), __uint_as_float(y[4 * q4 + 3]));
         }
     }
-    fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();
-    if (tid == 0) {
-        bulk_store(rec + kRecW, smem + kI_QK + 8192, 8192);
-        bulk_store(rec + kRecW + 8192, smem + kI_QK + 24576, 8192);
-        bulk_commit();
-        bulk_wait_read_all();
-    }
+    if (tid == 0) bulk_wait_read_all();
     if (warp == 0) tmem_dealloc(tmem, kIntraTmemCols);
 }
 

@@ -30,10 +30,10 @@ def run_prefill(p, impl, slot_idx=None, num_slots=None, init="from_inputs", alia
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     args = (U.dev_bf16(p["q"]), U.dev_bf16(p["k"]), U.dev_bf16(p["v"]), U.dev(p["g"]),
             U.dev(p["beta"]), U.dev(p["cu_seqlens"]), init_t, final, U.dev(slot_idx), o, p["scale"])
-    if impl == "chunked":
+    if impl in ("chunked", "auto"):
         ws = torch.empty(max(api.gdn_prefill_workspace_bytes(T, N, p["Hqk"], Hv), 256),
                          dtype=torch.uint8, device="cuda")
-        api.gdn_prefill(*args, ws, dev_status=status)
+        api.gdn_prefill(*args, ws, dev_status=status, route=impl)
     else:
         api.gdn_prefill_recurrent(*args, dev_status=status)
     torch.cuda.synchronize()
@@ -197,3 +197,12 @@ def test_chunked_repeatable_under_load_many_ctas():
     o_ref, S_ref, _ = oracle_prefill(p)
     U.check_o(ref_o, o_ref, U.O_REL_L2_PREFILL)
     U.check_state(ref_S.astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
+
+
+@pytest.mark.parametrize("lens", [[1], [6], [16], [3, 16, 0, 9], [17], [12, 35]])
+def test_length_routed_entry_point_small_shapes(lens):
+    """gdn_prefill itself (routing by length: up to 16 tokens per sequence the token-by-token
+    kernel, beyond that the chunked kernels) on the tiny shapes of the short-prompt regime."""
+    p = I.prefill_inputs(lens, 2, 4, seed=5000 + sum(lens), init="normal")
+    o, S, o_ref, S_ref = compare(p, "auto")
+    U.check_state(S.astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
