@@ -1,0 +1,492 @@
+// Device-side building blocks shared by the chunked prefill kernels (the three-launch path and
+// the fused single-launch path): shared-memory maps, the fp32 triangular solve, the intra-chunk
+// item routine, and the bounded-wait helpers.  See gdn_prefill_chunk.cuh for the algebra.
+#pragma once
+#include "gdn_prefill_chunk.cuh"
+#include "gdn_sm100.cuh"
+
+namespace gdn {
+using namespace sm100;
+
+constexpr int kIntraThreads = 256;
+constexpr uint32_t kIntraTmemCols = 128;
+constexpr int kLdA = 68;               // row stride (floats) of the fp32 A / T matrix
+// Shared memory map (bytes from a 1024-aligned base).  Regions are reused as their contents die
+// so that three CTAs fit on an SM:
+//   R1  Q/K tiles.  Q halves -> Qg image (stored early) -> T_w and T_u(hi);  K halves -> W image.
+//   R2  A, then T, in fp32 plus the solve scratch -> V tile (loaded after the solve).
+//   R3  P image (stored early) -> T_u(lo).
+constexpr uint32_t kI_QK = 0;          // 2 halves x [128 rows x 128 B]: rows 0-63 Q, 64-127 K
+constexpr uint32_t kI_Tw = 0;          // over Q half 0: T diag(beta e^b) [64 r x 64 i] bf16, K-major
+constexpr uint32_t kI_Tu = 16384;      // over Q half 1: T diag(beta) rounded to bf16 ...
+constexpr uint32_t kI_A = 32768;       // A, then T in place: fp32 [64][kLdA]
+constexpr uint32_t kI_Scr = kI_A + 64 * kLdA * 4;      // solve scratch, fp32 [32][40]
+constexpr uint32_t kI_V = 32768;       // over A: 2 halves x [64 x 128 B]
+constexpr uint32_t kI_P = 32768 + 22528;               // P image staging
+constexpr uint32_t kI_TuLo = kI_P;     // ... and the bf16 remainder of T diag(beta)
+constexpr uint32_t kI_End = kI_P + 8192;
+constexpr uint32_t kIntraSmem = kI_End + 1024;         // + alignment slack
+static_assert(kI_Scr + 32 * 40 * 4 <= kI_P, "solve scratch overlaps the P image");
+
+struct TensorMaps {
+    CUtensorMap q, k, v;
+};
+
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// One 16x8 output tile  C += A[16 x 8*ksteps] * B[8*ksteps x 8]  on mma.sync m16n8k8 with both
+// operands split into tf32 hi + lo parts (three products; the lo*lo term is dropped), which keeps
+// fp32-level accuracy.  A, B: fp32 row-major in shared memory; g = lane / 4, t = lane % 4.
+__device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo) {
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(hi) : "f"(x));
+    const float rem = x - __uint_as_float(hi);
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(lo) : "f"(rem));
+}
+__device__ __forceinline__ void mma_m16n8k8_tf32(float (&c)[4], const uint32_t (&a)[4],
+                                                 const uint32_t (&b)[2]) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+__device__ __forceinline__ void mma_tile_tf32x3(const float* A, int lda, const float* B, int ldb,
+                                                int ksteps, float (&c)[4], int g, int t) {
+    float c1[4] = {0.f, 0.f, 0.f, 0.f}, c2[4] = {0.f, 0.f, 0.f, 0.f};   // separate dependency chains
+#pragma unroll 4
+    for (int ks = 0; ks < ksteps; ++ks) {
+        const float* a_ = A + 8 * ks;
+        const float* b_ = B + (8 * ks) * ldb;
+        const float af[4] = {a_[g * lda + t], a_[(g + 8) * lda + t], a_[g * lda + t + 4],
+                             a_[(g + 8) * lda + t + 4]};
+        const float bf[2] = {b_[t * ldb + g], b_[(t + 4) * ldb + g]};
+        uint32_t ah[4], al[4], bh[2], bl[2];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) split_tf32(af[i], ah[i], al[i]);
+#pragma unroll
+        for (int i = 0; i < 2; ++i) split_tf32(bf[i], bh[i], bl[i]);
+        mma_m16n8k8_tf32(c1, al, bh);
+        mma_m16n8k8_tf32(c2, ah, bl);
+        mma_m16n8k8_tf32(c, ah, bh);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) c[i] += c1[i] + c2[i];
+}
+
+// T = (I + A)^{-1} for the strictly lower-triangular 64x64 A in sA (row-major, stride kLdA),
+// in place, by 256 threads: four 16x16 diagonal blocks by forward substitution in fp32, then the
+// off-diagonal blocks by block elimination at block sizes 16 and 32
+//     [[Ta, 0], [X, Tb]],  X = -Tb (A_ba Ta),
+// whose small products run on the legacy mma.sync path with split-tf32 operands (fp32-level
+// accuracy; tcgen05 needs M >= 64).  Ends with a __syncthreads().
+template <class Sync>
+__device__ __forceinline__ void solve_unit_lower_64(float* sA, float* scr, int tid, Sync sync) {
+    // ---- diagonal blocks: thread (I, j) computes column j of (I + A_II)^{-1}, right-looking
+    if (tid < 64) {
+        const int I = tid >> 4, j = tid & 15;
+        float* blk = sA + (16 * I) * kLdA + 16 * I;
+        float t[16];
+#pragma unroll
+        for (int r = 0; r < 16; ++r) t[r] = (r == j) ? 1.f : 0.f;
+#pragma unroll
+        for (int i = 0; i < 15; ++i) {
+            const float ti = t[i];
+#pragma unroll
+            for (int r = i + 1; r < 16; ++r) t[r] = fmaf(-blk[r * kLdA + i], ti, t[r]);
+        }
+        __syncwarp();                      // every column of the block has read A_II
+#pragma unroll
+        for (int r = 0; r < 16; ++r) blk[r * kLdA + j] = t[r];
+    }
+    sync();
+    // ---- off-diagonal blocks on the tensor cores (mma.sync m16n8k8, 3xTF32: fp32-level accuracy)
+    const int warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+    // 16-blocks (1,0) and (3,2): X = A_IJ T_JJ, then T_IJ = -T_II X.  Four 16x8 tiles, warps 0-3.
+    {
+        const int pr = warp >> 1, nb = warp & 1;            // pair, 8-column block
+        const int I = 2 * pr + 1, J = 2 * pr;
+        float* X = scr + pr * (16 * 24);
+        float c[4] = {0.f, 0.f, 0.f, 0.f};
+        if (warp < 4) {
+            mma_tile_tf32x3(sA + (16 * I) * kLdA + 16 * J, kLdA, sA + (16 * J) * kLdA + 16 * J + 8 * nb,
+                            kLdA, 2, c, g, t);
+            *reinterpret_cast<float2*>(X + g * 24 + 8 * nb + 2 * t) = make_float2(c[0], c[1]);
+            *reinterpret_cast<float2*>(X + (g + 8) * 24 + 8 * nb + 2 * t) = make_float2(c[2], c[3]);
+        }
+        sync();
+        if (warp < 4) {
+            c[0] = c[1] = c[2] = c[3] = 0.f;
+            mma_tile_tf32x3(sA + (16 * I) * kLdA + 16 * I, kLdA, X + 8 * nb, 24, 2, c, g, t);
+            float* dst = sA + (16 * I) * kLdA + 16 * J + 8 * nb;
+            *reinterpret_cast<float2*>(dst + g * kLdA + 2 * t) = make_float2(-c[0], -c[1]);
+            *reinterpret_cast<float2*>(dst + (g + 8) * kLdA + 2 * t) = make_float2(-c[2], -c[3]);
+        }
+    }
+    sync();
+    // 32-block (1,0): Y = A_ba Ta, then X = -Tb Y.  Eight 16x8 tiles, one per warp.
+    {
+        const int mr = warp >> 2, nb = warp & 3;
+        float c[4] = {0.f, 0.f, 0.f, 0.f};
+        mma_tile_tf32x3(sA + (32 + 16 * mr) * kLdA, kLdA, sA + 8 * nb, kLdA, 4, c, g, t);
+        *reinterpret_cast<float2*>(scr + (16 * mr + g) * 40 + 8 * nb + 2 * t) = make_float2(c[0], c[1]);
+        *reinterpret_cast<float2*>(scr + (16 * mr + g + 8) * 40 + 8 * nb + 2 * t) = make_float2(c[2], c[3]);
+        sync();
+        c[0] = c[1] = c[2] = c[3] = 0.f;
+        mma_tile_tf32x3(sA + (32 + 16 * mr) * kLdA + 32, kLdA, scr + 8 * nb, 40, 4, c, g, t);
+        float* dst = sA + (32 + 16 * mr) * kLdA + 8 * nb;
+        *reinterpret_cast<float2*>(dst + g * kLdA + 2 * t) = make_float2(-c[0], -c[1]);
+        *reinterpret_cast<float2*>(dst + (g + 8) * kLdA + 2 * t) = make_float2(-c[2], -c[3]);
+    }
+    sync();
+}
+
+// Lane 0 polls the mbarrier (bounded), the other lanes block at the warp barrier instead of
+// competing for issue slots; returns the same verdict on every lane.
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity) {
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity) ? 1 : 0;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+
+__device__ __forceinline__ uint32_t scale_bf16x2(uint32_t packed, float f) {
+    return pack_bf16(__uint_as_float(packed << 16) * f, __uint_as_float(packed & 0xffff0000u) * f);
+}
+
+// Per-group statics of the intra-chunk work (one instance per concurrently processed item).
+struct IntraStatics {
+    uint64_t bar_tma, bar_v, bar_mma;
+    int abort_flag;
+    int item;                          // work-queue slot (persistent variant)
+    alignas(16) float s_b2[kChunk];    // b_r log2(e): inclusive log-decay prefix
+    alignas(16) float s_beta[kChunk];  // beta_r (0 past the chunk's length)
+    alignas(16) float s_bg[kChunk];    // beta_r e^{b_r}
+    alignas(16) float s_eb[kChunk];    // e^{b_r}
+};
+
+// The intra-chunk quantities of one (chunk, v-head) item, computed by a group of 256 threads
+// (tid = 0..255 within the group; its warps must be CTA warps 0-3 mod 4 aligned, because a warp
+// reaches TMEM lanes 32 (warp % 4) ...).  `smem` is the group's 1024-aligned slice of kI_End
+// bytes, `tmem` its 128 TMEM columns, `sync` a barrier over exactly the group.  Writes the item's
+// record; returns false after a bounded wait gave up (status word set, nothing left in flight).
+template <class Sync>
+__device__ __forceinline__ bool intra_item(const TensorMaps& maps, const PrefillParams& p,
+                                           uint8_t* rec, const ChunkInfo ci, const int hqk,
+                                           const int hv, uint8_t* smem, IntraStatics& st,
+                                           const uint32_t tmem, const int tid, Sync sync) {
+    const int warp = tid >> 5;
+    const int colhalf = warp >> 2;                   // which 32 of the 64 accumulator columns
+    if (tid == 0) {
+        mbar_init(&st.bar_tma, 1);
+        mbar_init(&st.bar_v, 1);
+        mbar_init(&st.bar_mma, 1);
+        st.abort_flag = 0;
+        fence_barrier_init();
+        // Q and K first: everything below overlaps their flight (V comes later, over dead data)
+        mbar_expect_tx(&st.bar_tma, 32768);
+        tma_load_2d(smem + kI_QK, &maps.q, hqk * kD, ci.t0, &st.bar_tma);
+        tma_load_2d(smem + kI_QK + 8192, &maps.k, hqk * kD, ci.t0, &st.bar_tma);
+        tma_load_2d(smem + kI_QK + 16384, &maps.q, hqk * kD + 64, ci.t0, &st.bar_tma);
+        tma_load_2d(smem + kI_QK + 24576, &maps.k, hqk * kD + 64, ci.t0, &st.bar_tma);
+    }
+    if (warp == 1) {
+        // inclusive prefix sum of the log gates over the chunk (two tokens per lane); rows past
+        // the chunk's length get g = 0, beta = 0 and so change nothing downstream
+        const int lane = tid & 31;
+        float g0 = 0.f, g1 = 0.f, be0 = 0.f, be1 = 0.f;
+        if (2 * lane < ci.len) {
+            const size_t th = static_cast<size_t>(ci.t0 + 2 * lane) * p.Hv + hv;
+            g0 = p.g[th]; be0 = p.beta[th];
+        }
+        if (2 * lane + 1 < ci.len) {
+            const size_t th = static_cast<size_t>(ci.t0 + 2 * lane + 1) * p.Hv + hv;
+            g1 = p.g[th]; be1 = p.beta[th];
+        }
+        float incl = g0 + g1;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const float y = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += y;
+        }
+        const float kLog2e = 1.4426950408889634f;
+        const float b1 = incl, b0 = incl - g1;
+        const float bC = __shfl_sync(0xffffffffu, incl, 31);
+        st.s_b2[2 * lane] = b0 * kLog2e; st.s_b2[2 * lane + 1] = b1 * kLog2e;
+        st.s_beta[2 * lane] = be0; st.s_beta[2 * lane + 1] = be1;
+        const float e0 = ex2_approx(b0 * kLog2e), e1 = ex2_approx(b1 * kLog2e);
+        st.s_eb[2 * lane] = e0; st.s_eb[2 * lane + 1] = e1;
+        st.s_bg[2 * lane] = be0 * e0; st.s_bg[2 * lane + 1] = be1 * e1;
+        // decay vector of the record: e^{b_C - b_c}, then e^{b_C}
+        float* dec = reinterpret_cast<float*>(rec + kRecDecay);
+        dec[2 * lane] = ex2_approx((bC - b0) * kLog2e);
+        dec[2 * lane + 1] = ex2_approx((bC - b1) * kLog2e);
+        if (lane == 0) dec[kChunk] = ex2_approx(bC * kLog2e);
+    }
+    sync();
+    // On a timeout: flag it and let thread 0 drain what it has in flight; the caller unwinds.
+    auto bail = [&](bool stores_pending) {
+        if (tid == 0) {
+            report(p.dev_status, kDevTimeout);
+            if (stores_pending) bulk_wait_read_all();
+        }
+    };
+
+    if (warp == 0 && !warp_wait(&st.bar_tma, 0)) st.abort_flag = 1;      // one warp polls, the rest block
+    sync();
+    if (st.abort_flag) { bail(false); return false; }
+    tc_fence_after_sync();
+
+    const uint32_t tG = tmem, tW = tmem, tU = tmem + 64;     // W reuses the Gram columns
+    const uint32_t sQK = smem_u32(smem + kI_QK);
+    if (tid == 0) {
+        // [Q;K] (128 x 128, K-major) times K^T: lanes 0-63 = q.k, lanes 64-127 = k.k
+        const uint32_t idesc = make_idesc_bf16(128, 64, false, false);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
+            mma_ss(tG, make_sdesc_sw128(sQK + off, 16, 1024),
+                   make_sdesc_sw128(sQK + 8192 + off, 16, 1024), idesc, ks > 0);
+        }
+        mma_commit(&st.bar_mma);
+    }
+    if (warp == 0 && !warp_wait(&st.bar_mma, 0)) st.abort_flag = 1;
+    sync();
+    if (st.abort_flag) { bail(false); return false; }
+    tc_fence_after_sync();
+
+    const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    float* sA = reinterpret_cast<float*>(smem + kI_A);
+    {
+        // Accumulator row of this thread: TMEM lane 32 (warp % 4) + lane; lanes 0-63 hold q.k
+        // rows (-> P), lanes 64-127 hold k.k rows (-> A).  The thread covers 32 of the 64 columns,
+        // 16 at a time.
+        const int row = (warp & 3) * 32 + (tid & 31);
+        const int r = row & 63;
+        const bool is_p = row < 64;
+        const float br2 = st.s_b2[r];
+        const float rowscale = is_p ? 1.f : st.s_beta[r];
+        const int limit = is_p ? r : r - 1;              // keep columns i <= limit
+#pragma unroll
+        for (int step = 0; step < 2; ++step) {
+            const int cbase = colhalf * 32 + step * 16;
+            uint32_t x[16];
+            tmem_ld16(tG + lane_base + cbase, x);
+            tmem_wait_ld();
+            float val[16];
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+                const float4 bb = *reinterpret_cast<const float4*>(st.s_b2 + cbase + 4 * q4);
+                const float bv[4] = {bb.x, bb.y, bb.z, bb.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int jj = 4 * q4 + e;
+                    const bool keep = cbase + jj <= limit;
+                    const float dec = ex2_approx(keep ? br2 - bv[e] : 0.f);   // e^{b_r - b_i}
+                    val[jj] = keep ? rowscale * dec * __uint_as_float(x[jj]) : 0.f;
+                }
+            }
+            if (is_p) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint4 w;
+                    w.x = pack_bf16(val[8 * h + 0], val[8 * h + 1]);
+                    w.y = pack_bf16(val[8 * h + 2], val[8 * h + 3]);
+                    w.z = pack_bf16(val[8 * h + 4], val[8 * h + 5]);
+                    w.w = pack_bf16(val[8 * h + 6], val[8 * h + 7]);
+                    *reinterpret_cast<uint4*>(smem + kI_P + sw128_offset(r, (cbase >> 3) + h)) = w;
+                }
+            } else {
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4)
+                    *reinterpret_cast<float4*>(sA + r * kLdA + cbase + 4 * q4) =
+                        make_float4(val[4 * q4], val[4 * q4 + 1], val[4 * q4 + 2], val[4 * q4 + 3]);
+            }
+        }
+    }
+    {   // Q rows scaled by e^{b_r}, in place (the Gram product has consumed Q): this is the Qg image
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const int idx = tid + it * kIntraThreads;          // 1024 16-byte pieces
+            const int halfq = idx >> 9, rem = idx & 511;
+            const int r = rem >> 3;
+            uint4* ptr = reinterpret_cast<uint4*>(smem + kI_QK + halfq * 16384 + rem * 16);
+            const float f = st.s_eb[r];
+            uint4 w = *ptr;
+            w.x = scale_bf16x2(w.x, f); w.y = scale_bf16x2(w.y, f);
+            w.z = scale_bf16x2(w.z, f); w.w = scale_bf16x2(w.w, f);
+            *ptr = w;
+        }
+    }
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    sync();
+    if (tid == 0) {
+        // Qg and P are final: store them now; their shared memory is reused after the solve
+        bulk_store(rec + kRecQg, smem + kI_QK, 8192);
+        bulk_store(rec + kRecQg + 8192, smem + kI_QK + 16384, 8192);
+        bulk_store(rec + kRecP, smem + kI_P, 8192);
+        bulk_commit();
+    }
+
+    solve_unit_lower_64(sA, reinterpret_cast<float*>(smem + kI_Scr), tid, sync);
+
+    if (tid == 0) bulk_wait_read_all();      // the Q halves and the P image have been read out
+    sync();
+
+    {   // T (fp32, row-major) -> bf16 B operands T diag(beta e^b), T diag(beta) (hi, lo)
+#pragma unroll
+        for (int it = 0; it < 2; ++it) {
+            const int idx = tid + it * kIntraThreads;          // 512 pieces of 8 columns
+            const int r = idx >> 3, c8 = idx & 7;
+            const float4 t0 = *reinterpret_cast<const float4*>(sA + r * kLdA + 8 * c8);
+            const float4 t1 = *reinterpret_cast<const float4*>(sA + r * kLdA + 8 * c8 + 4);
+            const float4 g0 = *reinterpret_cast<const float4*>(st.s_bg + 8 * c8);
+            const float4 g1 = *reinterpret_cast<const float4*>(st.s_bg + 8 * c8 + 4);
+            const float4 e0 = *reinterpret_cast<const float4*>(st.s_beta + 8 * c8);
+            const float4 e1 = *reinterpret_cast<const float4*>(st.s_beta + 8 * c8 + 4);
+            const float tv[8] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+            const float gv[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+            const float ev[8] = {e0.x, e0.y, e0.z, e0.w, e1.x, e1.y, e1.z, e1.w};
+            uint32_t w[4], hi[4], lo[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                w[j] = pack_bf16(tv[2 * j] * gv[2 * j], tv[2 * j + 1] * gv[2 * j + 1]);
+                const float u0 = tv[2 * j] * ev[2 * j], u1 = tv[2 * j + 1] * ev[2 * j + 1];
+                hi[j] = pack_bf16(u0, u1);
+                lo[j] = pack_bf16(u0 - __uint_as_float(hi[j] << 16),
+                                  u1 - __uint_as_float(hi[j] & 0xffff0000u));
+            }
+            const uint32_t off = sw128_offset(r, c8);
+            *reinterpret_cast<uint4*>(smem + kI_Tw + off) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4*>(smem + kI_Tu + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            *reinterpret_cast<uint4*>(smem + kI_TuLo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        }
+    }
+    fence_proxy_async_smem();
+    sync();
+
+    const uint32_t sV = smem_u32(smem + kI_V);
+    if (tid == 0) {
+        // V into the space the solve has left; meanwhile W^T (dk x r) = K^T T_w^T with the raw K
+        // tile read MN-major
+        mbar_expect_tx(&st.bar_v, 16384);
+        tma_load_2d(smem + kI_V, &maps.v, hv * kD, ci.t0, &st.bar_v);
+        tma_load_2d(smem + kI_V + 8192, &maps.v, hv * kD + 64, ci.t0, &st.bar_v);
+        const uint32_t idesc = make_idesc_bf16(128, 64, true, false);
+        const uint32_t sTw = smem_u32(smem + kI_Tw);
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+            mma_ss(tW, make_sdesc_sw128(sQK + 8192 + ks * 2048, 16384, 1024),
+                   make_sdesc_sw128(sTw + ks * 32, 16, 1024), idesc, ks > 0);
+        mma_commit(&st.bar_mma);
+    }
+    if (warp == 0 && !warp_wait(&st.bar_mma, 1)) st.abort_flag = 1;
+    sync();
+    if (st.abort_flag) { bail(false); return false; }      // nothing of thread 0's stores is pending here
+    tc_fence_after_sync();
+
+    const int d = (warp & 3) * 32 + (tid & 31);   // TMEM lane of this thread: a dk / dv index
+    {   // W^T[d][32 tokens] -> bf16 -> W image staged over the (now dead) K halves
+        uint8_t* sW = smem + kI_QK + 8192 + (d >> 6) * 16384;
+        const uint32_t wcol = ((d & 7) << 1);
+        const uint32_t wchunk = (d & 63) >> 3;
+#pragma unroll
+        for (int step = 0; step < 2; ++step) {
+            const int cbase = colhalf * 32 + step * 16;
+            uint32_t x[16];
+            tmem_ld16(tW + lane_base + cbase, x);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                *reinterpret_cast<__nv_bfloat16*>(sW + sw128_offset(cbase + j, wchunk) + wcol) =
+                    __float2bfloat16(__uint_as_float(x[j]));
+        }
+    }
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    if (warp == 0 && !warp_wait(&st.bar_v, 0)) st.abort_flag = 1;        // V has landed
+    sync();
+    if (st.abort_flag) { bail(false); return false; }
+    tc_fence_after_sync();
+    if (tid == 0) {
+        bulk_store(rec + kRecW, smem + kI_QK + 8192, 8192);
+        bulk_store(rec + kRecW + 8192, smem + kI_QK + 24576, 8192);
+        bulk_commit();
+        // U~^T (dv x r) = V^T T_u^T with T_u = hi + lo
+        const uint32_t idesc = make_idesc_bf16(128, 64, true, false);
+        const uint32_t sTu = smem_u32(smem + kI_Tu), sTuLo = smem_u32(smem + kI_TuLo);
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+            mma_ss(tU, make_sdesc_sw128(sV + ks * 2048, 8192, 1024),
+                   make_sdesc_sw128(sTu + ks * 32, 16, 1024), idesc, ks > 0);
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+            mma_ss(tU, make_sdesc_sw128(sV + ks * 2048, 8192, 1024),
+                   make_sdesc_sw128(sTuLo + ks * 32, 16, 1024), idesc, true);
+        mma_commit(&st.bar_mma);
+    }
+    if (warp == 0 && !warp_wait(&st.bar_mma, 0)) st.abort_flag = 1;
+    sync();
+    if (st.abort_flag) { bail(true); return false; }
+    tc_fence_after_sync();
+
+    {   // U~^T[d][32 tokens] -> record, [token group][dv][4 tokens] fp32
+        float4* urec = reinterpret_cast<float4*>(rec + kRecU);
+#pragma unroll
+        for (int step = 0; step < 2; ++step) {
+            const int cbase = colhalf * 32 + step * 16;
+            uint32_t y[16];
+            tmem_ld16(tU + lane_base + cbase, y);
+            tmem_wait_ld();
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4)
+                urec[((cbase >> 2) + q4) * kD + d] =
+                    make_float4(__uint_as_float(y[4 * q4]), __uint_as_float(y[4 * q4 + 1]),
+                                __uint_as_float(y[4 * q4 + 2]), __uint_as_float(y[4 * q4 + 3]));
+        }
+    }
+    tc_fence_before_sync();
+    sync();
+    if (tid == 0) bulk_wait_read_all();
+    return true;
+}
+
+constexpr int kStateEpiWarps = 8;
+constexpr int kStateEpiThreads = kStateEpiWarps * 32;
+constexpr int kStateThreads = kStateEpiThreads + 32;
+constexpr uint32_t kStateTmemCols = 512;
+constexpr uint32_t kS_Rec = 0;                 // record image (74240 B, padded to 74752)
+constexpr uint32_t kS_K = 74752;               // K tile, 2 halves [64 x 128 B]
+constexpr uint32_t kStageBytes = 74752 + 16384;                 // 91136
+constexpr uint32_t kS_Out = 2 * kStageBytes;   // o staging [64 tokens][128 dv] bf16
+constexpr uint32_t kStateSmem = 2 * kStageBytes + 16384 + 1024;
+// TMEM columns
+constexpr uint32_t kT_D1 = 0, kT_Y = 64 /* two tiles of 64 */, kT_D4 = 192, kT_S = 320, kT_U = 384,
+                   kT_Us = 416, kT_UsLo = 448;
+
+// bounded wait that also gives up as soon as another role has flagged an abort
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 255u) == 255u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+// Same, for a whole warp: lane 0 polls, every lane gets the verdict.
+__device__ __forceinline__ bool warp_wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = wait_or_abort(bar, parity, abort_flag) ? 1 : 0;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+
+__device__ __forceinline__ void epi_group_sync() {      // the 256 epilogue threads only
+    asm volatile("bar.sync 1, %0;" ::"n"(kStateEpiThreads) : "memory");
+}
+
+
+}  // namespace gdn
