@@ -96,13 +96,13 @@ int gdn_prefill_recurrent(const void* q, const void* k, const void* v, const flo
     return cuda_status(gdn::launch_prefill_recurrent(p, static_cast<cudaStream_t>(stream)));
 }
 
-int gdn_prefill_chunked(const void* q, const void* k, const void* v, const float* g,
-                        const float* beta, const int32_t* cu_seqlens, const float* init_state,
-                        float* final_state, const int32_t* slot_idx, void* o, int32_t T, int32_t N,
-                        int32_t max_seqlen_hint, int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv,
-                        int32_t chunk, int32_t num_slots, float scale, void* workspace,
-                        size_t workspace_bytes, int32_t* dev_status, void* stream) {
-    (void)max_seqlen_hint;
+namespace {
+int prefill_chunked_impl(bool fused, const void* q, const void* k, const void* v, const float* g,
+                         const float* beta, const int32_t* cu_seqlens, const float* init_state,
+                         float* final_state, const int32_t* slot_idx, void* o, int32_t T, int32_t N,
+                         int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv, int32_t chunk,
+                         int32_t num_slots, float scale, void* workspace, size_t workspace_bytes,
+                         int32_t* dev_status, void* stream) {
     if (chunk != gdn::kChunk) return GDN_ERR_SHAPE;
     const int rc = check_prefill(q, k, v, g, beta, cu_seqlens, init_state, final_state, o,
                                  T, N, Hqk, Hv, dk, dv, num_slots);
@@ -123,7 +123,33 @@ int gdn_prefill_chunked(const void* q, const void* k, const void* v, const float
     p.dev_status = dev_status;
     cp.ws = static_cast<uint8_t*>(workspace);
     cp.lay = gdn::workspace_layout(T, N, Hv);
-    return cuda_status(gdn::launch_prefill_chunked(cp, static_cast<cudaStream_t>(stream)));
+    return cuda_status(fused ? gdn::launch_prefill_fused(cp, static_cast<cudaStream_t>(stream))
+                             : gdn::launch_prefill_chunked(cp, static_cast<cudaStream_t>(stream)));
+}
+}  // namespace
+
+int gdn_prefill_chunked(const void* q, const void* k, const void* v, const float* g,
+                        const float* beta, const int32_t* cu_seqlens, const float* init_state,
+                        float* final_state, const int32_t* slot_idx, void* o, int32_t T, int32_t N,
+                        int32_t max_seqlen_hint, int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv,
+                        int32_t chunk, int32_t num_slots, float scale, void* workspace,
+                        size_t workspace_bytes, int32_t* dev_status, void* stream) {
+    (void)max_seqlen_hint;
+    return prefill_chunked_impl(false, q, k, v, g, beta, cu_seqlens, init_state, final_state,
+                                slot_idx, o, T, N, Hqk, Hv, dk, dv, chunk, num_slots, scale,
+                                workspace, workspace_bytes, dev_status, stream);
+}
+
+int gdn_prefill_fused(const void* q, const void* k, const void* v, const float* g,
+                      const float* beta, const int32_t* cu_seqlens, const float* init_state,
+                      float* final_state, const int32_t* slot_idx, void* o, int32_t T, int32_t N,
+                      int32_t max_seqlen_hint, int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv,
+                      int32_t chunk, int32_t num_slots, float scale, void* workspace,
+                      size_t workspace_bytes, int32_t* dev_status, void* stream) {
+    (void)max_seqlen_hint;
+    return prefill_chunked_impl(true, q, k, v, g, beta, cu_seqlens, init_state, final_state,
+                                slot_idx, o, T, N, Hqk, Hv, dk, dv, chunk, num_slots, scale,
+                                workspace, workspace_bytes, dev_status, stream);
 }
 
 int gdn_prefill(const void* q, const void* k, const void* v, const float* g, const float* beta,

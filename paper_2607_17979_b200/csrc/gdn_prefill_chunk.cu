@@ -321,21 +321,26 @@ prefill_state_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
             store_state_bf16();
             hand_over(&bar_s);
             bool ok = true;
+            auto await = [&](uint64_t* bar, uint32_t parity) {   // bounded wait + tcgen05 fence
+                if (ok && !warp_wait_or_abort(bar, parity, abortp)) ok = false;
+                tc_fence_after_sync();
+            };
             for (int j = 0; j < nc; ++j) {
                 const int st = j & 1;
                 const uint8_t* base = smem + st * kStageBytes;
+                // Every warp runs every group barrier and hand-over of every iteration, also after a
+                // wait has failed (ok == false: later waits and all work are skipped), so that no
+                // warp is ever left alone at a barrier.
                 if (j > 0) {     // part A of the previous chunk's outputs, while D1 is in flight
-                    if (!warp_wait_or_abort(&bar_y, (j - 1) & 1, abortp)) { ok = false; break; }
-                    tc_fence_after_sync();
+                    await(&bar_y, (j - 1) & 1);
                     epi_group_sync();
-                    outputs_stage(j - 1);
+                    if (ok) outputs_stage(j - 1);
                 }
-                if (!warp_wait_or_abort(&bar_full[st], (j >> 1) & 1, abortp)) { ok = false; break; }
-                if (!warp_wait_or_abort(&bar_d1, j & 1, abortp)) { ok = false; break; }
-                tc_fence_after_sync();
+                await(&bar_full[st], (j >> 1) & 1);
+                await(&bar_d1, j & 1);
 
                 const float* sdec = reinterpret_cast<const float*>(base + kS_Rec + kRecDecay);
-                {   // U^T[dv][c] = U~^T - D1 for the thread's 32 tokens [32*half, 32*half+32)
+                if (ok) {   // U^T[dv][c] = U~^T - D1 for the thread's 32 tokens [32*half, 32*half+32)
                     const float4* sU = reinterpret_cast<const float4*>(base + kS_Rec + kRecU);
                     uint32_t xa[16], xb[16];
                     tmem_ld16(tmem + kT_D1 + lane_base + half * 32, xa);
@@ -378,12 +383,11 @@ prefill_state_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
                 hand_over(&bar_u);
                 if (j > 0) {     // part B, while this chunk's state product is in flight
                     epi_group_sync();
-                    outputs_flush(j - 1);
+                    if (ok) outputs_flush(j - 1);
                 }
 
-                if (!warp_wait_or_abort(&bar_d4, j & 1, abortp)) { ok = false; break; }
-                tc_fence_after_sync();
-                {   // S <- e^{b_C} S + D4 on the thread's 64 dk columns; refresh the bf16 copy
+                await(&bar_d4, j & 1);
+                if (ok) {   // S <- e^{b_C} S + D4 on the thread's 64 dk columns; refresh the bf16 copy
                     const float gC = reinterpret_cast<const float*>(base + kS_Rec + kRecGammaC)[0];
 #pragma unroll
                     for (int c0 = 0; c0 < 64; c0 += 32) {
@@ -401,15 +405,11 @@ prefill_state_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
                 }
                 hand_over(&bar_s);
             }
-            if (ok) {
-                if (warp_wait_or_abort(&bar_y, (nc - 1) & 1, abortp)) {
-                    tc_fence_after_sync();
-                    epi_group_sync();
-                    outputs_stage(nc - 1);
-                    epi_group_sync();
-                    outputs_flush(nc - 1);
-                }
-            }
+            await(&bar_y, (nc - 1) & 1);
+            epi_group_sync();
+            if (ok) outputs_stage(nc - 1);
+            epi_group_sync();
+            if (ok) outputs_flush(nc - 1);
         }
         tc_fence_before_sync();
         __syncthreads();
@@ -471,6 +471,12 @@ bool make_token_map(CUtensorMap* m, const void* base, int64_t rows, int64_t cols
 
 }  // namespace
 
+bool make_prefill_tensor_maps(TensorMaps* maps, const PrefillParams& p) {
+    return make_token_map(&maps->q, p.q, p.T, static_cast<int64_t>(p.Hqk) * kD) &&
+           make_token_map(&maps->k, p.k, p.T, static_cast<int64_t>(p.Hqk) * kD) &&
+           make_token_map(&maps->v, p.v, p.T, static_cast<int64_t>(p.Hv) * kD);
+}
+
 cudaError_t launch_prefill_chunked(const ChunkedParams& cp, cudaStream_t stream) {
     const PrefillParams& p = cp.p;
     cudaError_t e = cudaFuncSetAttribute(prefill_intra_kernel,
@@ -480,10 +486,7 @@ cudaError_t launch_prefill_chunked(const ChunkedParams& cp, cudaStream_t stream)
                              kStateSmem);
     if (e != cudaSuccess) return e;
     TensorMaps maps;
-    if (!make_token_map(&maps.q, p.q, p.T, static_cast<int64_t>(p.Hqk) * kD) ||
-        !make_token_map(&maps.k, p.k, p.T, static_cast<int64_t>(p.Hqk) * kD) ||
-        !make_token_map(&maps.v, p.v, p.T, static_cast<int64_t>(p.Hv) * kD))
-        return cudaErrorInvalidValue;
+    if (!make_prefill_tensor_maps(&maps, p)) return cudaErrorInvalidValue;
 
     prefill_prep_kernel<<<1, kPrepThreads, 0, stream>>>(p.cu_seqlens, p.T, p.N, cp.ws, cp.lay,
                                                         p.dev_status);

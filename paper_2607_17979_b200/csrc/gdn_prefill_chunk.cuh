@@ -45,26 +45,48 @@ struct ChunkInfo {      // 16 bytes
 };
 
 // Workspace layout (all offsets multiples of 256 bytes):
-//   [0,256)                      int32 total_chunks
+//   [0,256)                      int32 header: [0] total_chunks, [1] total_items
+//                                (= total_chunks * Hv), [2] item queue head, [3] unit queue head
 //   seq_first[N+1]               int32: first chunk of each sequence (prefix sum); an invalid
 //                                sequence has zero chunks and seq_bad[n] = 1
 //   seq_bad[N]                   int32
 //   chunks[max_chunks]           ChunkInfo
+//   -- used by the fused single-launch path only --
+//   seq_by_rank[N]               int32: sequences sorted by chunk count, longest first
+//   order[max_chunks]            int32: chunk ids in processing order: by position inside the
+//                                sequence first, by sequence rank second (so that the records
+//                                every state-pass unit needs next are produced first)
+//   hist, fill, cnt, pos[max_nc+2]  int32 scratch of the counting sort (max_nc = T/64 + 1)
+//   flags[max_chunks][Hv]        uint32: 1 once the record is complete and visible
+//   -- both paths --
 //   records[max_chunks][Hv]      kRecBytes each
 struct WorkspaceLayout {
-    size_t seq_first, seq_bad, chunks, records, total;
-    int32_t max_chunks;
+    size_t seq_first, seq_bad, chunks, seq_by_rank, order, hist, fill, cnt, pos, flags, records,
+        total;
+    int32_t max_chunks, max_nc;
 };
+
+constexpr int kHdrTotalChunks = 0, kHdrTotalItems = 1, kHdrItemHead = 2, kHdrUnitHead = 3;
 
 inline size_t round256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 
 inline WorkspaceLayout workspace_layout(int32_t T, int32_t N, int32_t Hv) {
     WorkspaceLayout w;
     w.max_chunks = T / kChunk + N;
+    w.max_nc = T / kChunk + 1;
+    const size_t nchunks = static_cast<size_t>(w.max_chunks ? w.max_chunks : 1);
+    const size_t nbins = round256(sizeof(int32_t) * (static_cast<size_t>(w.max_nc) + 2));
     w.seq_first = 256;
     w.seq_bad = w.seq_first + round256(sizeof(int32_t) * (static_cast<size_t>(N) + 1));
     w.chunks = w.seq_bad + round256(sizeof(int32_t) * static_cast<size_t>(N ? N : 1));
-    w.records = w.chunks + round256(sizeof(ChunkInfo) * static_cast<size_t>(w.max_chunks ? w.max_chunks : 1));
+    w.seq_by_rank = w.chunks + round256(sizeof(ChunkInfo) * nchunks);
+    w.order = w.seq_by_rank + round256(sizeof(int32_t) * static_cast<size_t>(N ? N : 1));
+    w.hist = w.order + round256(sizeof(int32_t) * nchunks);
+    w.fill = w.hist + nbins;
+    w.cnt = w.fill + nbins;
+    w.pos = w.cnt + nbins;
+    w.flags = w.pos + nbins;
+    w.records = w.flags + round256(sizeof(uint32_t) * nchunks * Hv);
     w.total = w.records + static_cast<size_t>(w.max_chunks) * Hv * kRecBytes;
     return w;
 }
@@ -76,5 +98,7 @@ struct ChunkedParams {
 };
 
 cudaError_t launch_prefill_chunked(const ChunkedParams& cp, cudaStream_t stream);
+// One cooperative launch: some CTAs produce the records, the others run the state pass behind them.
+cudaError_t launch_prefill_fused(const ChunkedParams& cp, cudaStream_t stream);
 
 }  // namespace gdn

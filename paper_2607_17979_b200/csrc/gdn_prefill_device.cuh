@@ -31,6 +31,8 @@ static_assert(kI_Scr + 32 * 40 * 4 <= kI_P, "solve scratch overlaps the P image"
 struct TensorMaps {
     CUtensorMap q, k, v;
 };
+// Host side: 2-D maps over the packed q, k, v (64 x 64 boxes, 128B swizzle); false on failure.
+bool make_prefill_tensor_maps(TensorMaps* maps, const PrefillParams& p);
 
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
@@ -176,15 +178,23 @@ template <class Sync>
 __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const PrefillParams& p,
                                            uint8_t* rec, const ChunkInfo ci, const int hqk,
                                            const int hv, uint8_t* smem, IntraStatics& st,
-                                           const uint32_t tmem, const int tid, Sync sync) {
+                                           const uint32_t tmem, const int tid, Sync sync,
+                                           const uint32_t n_done = 0) {
+    // `n_done` = items this group has processed before (persistent callers): the mbarriers are
+    // initialised once and keep flipping phase, one completion of bar_tma and bar_v and three
+    // of bar_mma per item.
+    const uint32_t par1 = n_done & 1u;           // parity of this item's bar_tma / bar_v phase
+    const uint32_t par3 = (3u * n_done) & 1u;    // parity of this item's first bar_mma phase
     const int warp = tid >> 5;
     const int colhalf = warp >> 2;                   // which 32 of the 64 accumulator columns
     if (tid == 0) {
-        mbar_init(&st.bar_tma, 1);
-        mbar_init(&st.bar_v, 1);
-        mbar_init(&st.bar_mma, 1);
+        if (n_done == 0) {
+            mbar_init(&st.bar_tma, 1);
+            mbar_init(&st.bar_v, 1);
+            mbar_init(&st.bar_mma, 1);
+            fence_barrier_init();
+        }
         st.abort_flag = 0;
-        fence_barrier_init();
         // Q and K first: everything below overlaps their flight (V comes later, over dead data)
         mbar_expect_tx(&st.bar_tma, 32768);
         tma_load_2d(smem + kI_QK, &maps.q, hqk * kD, ci.t0, &st.bar_tma);
@@ -234,7 +244,7 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
         }
     };
 
-    if (warp == 0 && !warp_wait(&st.bar_tma, 0)) st.abort_flag = 1;      // one warp polls, the rest block
+    if (warp == 0 && !warp_wait(&st.bar_tma, par1)) st.abort_flag = 1;      // one warp polls, the rest block
     sync();
     if (st.abort_flag) { bail(false); return false; }
     tc_fence_after_sync();
@@ -252,7 +262,7 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
         }
         mma_commit(&st.bar_mma);
     }
-    if (warp == 0 && !warp_wait(&st.bar_mma, 0)) st.abort_flag = 1;
+    if (warp == 0 && !warp_wait(&st.bar_mma, par3)) st.abort_flag = 1;
     sync();
     if (st.abort_flag) { bail(false); return false; }
     tc_fence_after_sync();
@@ -383,7 +393,7 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
                    make_sdesc_sw128(sTw + ks * 32, 16, 1024), idesc, ks > 0);
         mma_commit(&st.bar_mma);
     }
-    if (warp == 0 && !warp_wait(&st.bar_mma, 1)) st.abort_flag = 1;
+    if (warp == 0 && !warp_wait(&st.bar_mma, par3 ^ 1u)) st.abort_flag = 1;
     sync();
     if (st.abort_flag) { bail(false); return false; }      // nothing of thread 0's stores is pending here
     tc_fence_after_sync();
@@ -407,7 +417,7 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
     }
     fence_proxy_async_smem();
     tc_fence_before_sync();
-    if (warp == 0 && !warp_wait(&st.bar_v, 0)) st.abort_flag = 1;        // V has landed
+    if (warp == 0 && !warp_wait(&st.bar_v, par1)) st.abort_flag = 1;        // V has landed
     sync();
     if (st.abort_flag) { bail(false); return false; }
     tc_fence_after_sync();
@@ -428,7 +438,7 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
                    make_sdesc_sw128(sTuLo + ks * 32, 16, 1024), idesc, true);
         mma_commit(&st.bar_mma);
     }
-    if (warp == 0 && !warp_wait(&st.bar_mma, 0)) st.abort_flag = 1;
+    if (warp == 0 && !warp_wait(&st.bar_mma, par3)) st.abort_flag = 1;
     sync();
     if (st.abort_flag) { bail(true); return false; }
     tc_fence_after_sync();
