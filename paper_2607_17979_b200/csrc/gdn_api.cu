@@ -178,9 +178,18 @@ int gdn_prefill(const void* q, const void* k, const void* v, const float* g, con
                                      slot_idx, o, T, N, Hqk, Hv, dk, dv, num_slots, scale,
                                      dev_status, stream);
     }
-    return gdn_prefill_chunked(q, k, v, g, beta, cu_seqlens, init_state, final_state, slot_idx, o,
-                               T, N, max_seqlen_hint, Hqk, Hv, dk, dv, chunk, num_slots, scale,
-                               workspace, workspace_bytes, dev_status, stream);
+    // Few (sequence, v-head) units: the serial state pass would occupy only a few SMs while the
+    // rest idle, so run it next to the record producers in one cooperative launch.  Many units:
+    // the three-launch path keeps every SM on one kind of work at a time and is faster.
+    int dev = 0, sms = 148, coop = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) {
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+    }
+    const bool few_units = static_cast<long long>(N) * Hv <= sms / 3 && longest > 16 * gdn::kChunk;
+    return prefill_chunked_impl(coop && few_units, q, k, v, g, beta, cu_seqlens, init_state,
+                                final_state, slot_idx, o, T, N, Hqk, Hv, dk, dv, chunk, num_slots,
+                                scale, workspace, workspace_bytes, dev_status, stream);
 }
 
 const char* gdn_status_string(int code) {
