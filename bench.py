@@ -178,15 +178,11 @@ def run_reference(args):
 
 def run_ours(args):
     import torch
-    import torch.distributed as dist
-    from paper_2607_17979_b200 import api
+    from paper_2607_17979_b200 import api, dist as D
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = D.world()
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    D.init("nccl", torch.device("cuda", local))
 
     def bf16(bits):
         return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
@@ -216,12 +212,15 @@ def run_ours(args):
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     counter = {"step": 0}
 
-    # pinned host copies for the end-to-end leg
+    # pinned host buffers + device staging for the end-to-end leg (host-buffer entry points)
     h_dec = {n: t.cpu().pin_memory() for n, t in d_in.items()}
     h_do = torch.empty_like(d_o, device="cpu").pin_memory()
     h_pre = {n: t.cpu().pin_memory() for n, t in p_in.items()}
     h_cu = cu.cpu().pin_memory()
     h_po = torch.empty_like(p_o, device="cpu").pin_memory()
+    stage_d = torch.empty(api.gdn_decode_host_staging_bytes(B, Hqk, Hv), dtype=torch.uint8, device="cuda")
+    stage_p = torch.empty(api.gdn_prefill_host_staging_bytes(T, N, Hqk, Hv), dtype=torch.uint8,
+                          device="cuda")
 
     def decode_call():
         pool = pools[counter["step"] % DEC_POOLS]
@@ -249,24 +248,20 @@ def run_ours(args):
         counter["step"] += 1
         e0, e1, e2, e3 = ev(), ev(), ev(), ev()
         e0.record()
-        for n in d_in:
-            d_in[n].copy_(h_dec[n], non_blocking=True)
-        decode_call()
-        h_do.copy_(d_o, non_blocking=True)
+        api.gdn_decode_host(h_dec["q"], h_dec["k"], h_dec["v"], h_dec["g"], h_dec["beta"],
+                            pools[counter["step"] % DEC_POOLS], None, h_do, dec["scale"], stage_d,
+                            dev_status=status)
         e1.record()
         e2.record()
-        for n in p_in:
-            p_in[n].copy_(h_pre[n], non_blocking=True)
-        cu.copy_(h_cu, non_blocking=True)
-        prefill_call(p_in)
-        h_po.copy_(p_o, non_blocking=True)
+        api.gdn_prefill_host(h_pre["q"], h_pre["k"], h_pre["v"], h_pre["g"], h_pre["beta"], h_cu,
+                             None, p_final, None, h_po, pre["scale"], stage_p, ws,
+                             max_seqlen_hint=max(pre["seq_lens"]), dev_status=status)
         e3.record()
         if timed is not None:
             timed.append((e0, e1, e2, e3))
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        D.barrier()
         torch.cuda.synchronize()
 
     def timed_region(fn):
@@ -279,10 +274,8 @@ def run_ours(args):
         barrier()
         dec_ms = np.array([a.elapsed_time(b) for a, b, _, _ in evs])
         pre_ms = np.array([c.elapsed_time(d) for _, _, c, d in evs])
-        t = torch.tensor([dec_ms.mean(), pre_ms.mean()], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t[0]), float(t[1])
+        slowest = D.max_over_ranks([dec_ms.mean(), pre_ms.mean()], device="cuda")
+        return slowest[0], slowest[1]
 
     # clocks are sampled from before the warm-up to after the timed steps (the GPU is under the
     # same load throughout; the timed steps alone can be shorter than one sampling period)
@@ -341,14 +334,14 @@ def run_ours(args):
                              "kind": "oracle", "sample": cpu["sample"]},
             "e2e": {"value": world * state_b / (e2e_dec_ms * 1e-3) / 1e9, "unit": "GB/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": h_do.numel() * 2,
-                    "note": "q,k,v,g,beta from pinned host memory and o back each step; the state "
-                            "pool is the resident recurrent cache and stays in HBM"},
+                    "note": "gdn_decode_host / gdn_prefill_host: q,k,v,g,beta(,cu_seqlens) from pinned "
+                            "host memory and o back every step; the state pool is the resident "
+                            "recurrent cache and stays in HBM"},
             "gpu_launches": args.steps * api.LAUNCHES_PER_STEP,
             "clocks": clocks,
         }
         print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    D.finish()
 
 
 def main():

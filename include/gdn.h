@@ -213,6 +213,37 @@ int gdn_prefill_static(const void* q, const void* k, const void* v,
                        int32_t num_slots, float scale,
                        int32_t* dev_status, void* stream);
 
+/*
+ * Host-buffer variants (same operators; the paper has no counterpart: they are
+ * the end-to-end form a caller without device tensors uses).  q, k, v, g, beta,
+ * slot_idx / cu_seqlens and o are HOST pointers (pinned memory makes the copies
+ * asynchronous); state_pool / init_state / final_state, staging, workspace and
+ * dev_status stay DEVICE pointers.  The call enqueues the host->device copies
+ * into `staging` (at least gdn_*_host_staging_bytes(...), 256-byte aligned),
+ * the kernels, and the device->host copy of o on `stream`, and returns; o is
+ * valid once the stream has been synchronised.  Errors as the device variants,
+ * GDN_ERR_WORKSPACE also for a staging buffer that is too small.
+ */
+size_t gdn_decode_host_staging_bytes(int32_t B, int32_t Hqk, int32_t Hv);
+int gdn_decode_host(const void* q, const void* k, const void* v,
+                    const float* g, const float* beta,
+                    float* state_pool, const int32_t* slot_idx, void* o,
+                    int32_t B, int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv,
+                    int32_t num_slots, float scale,
+                    void* staging, size_t staging_bytes,
+                    int32_t* dev_status, void* stream);
+size_t gdn_prefill_host_staging_bytes(int32_t T, int32_t N, int32_t Hqk, int32_t Hv);
+int gdn_prefill_host(const void* q, const void* k, const void* v,
+                     const float* g, const float* beta, const int32_t* cu_seqlens,
+                     const float* init_state, float* final_state, const int32_t* slot_idx,
+                     void* o,
+                     int32_t T, int32_t N, int32_t max_seqlen_hint,
+                     int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv, int32_t chunk,
+                     int32_t num_slots, float scale,
+                     void* staging, size_t staging_bytes,
+                     void* workspace, size_t workspace_bytes,
+                     int32_t* dev_status, void* stream);
+
 /* Human-readable name of a return code (static storage, never NULL). */
 const char* gdn_status_string(int code);
 

@@ -16,7 +16,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libgdn_b200.so")
 
 EXPORTS = ("gdn_decode", "gdn_prefill_workspace_bytes", "gdn_prefill", "gdn_prefill_chunked",
-           "gdn_prefill_fused",
+           "gdn_prefill_fused", "gdn_decode_host", "gdn_decode_host_staging_bytes",
+           "gdn_prefill_host", "gdn_prefill_host_staging_bytes",
            "gdn_prefill_recurrent",
            "gdn_prefill_static", "gdn_prefill_static_workspace_bytes", "gdn_status_string",
            "gdn_last_cuda_error_string", "gdn_version")
@@ -49,6 +50,14 @@ _lib.gdn_prefill_static.restype = ctypes.c_int
 _lib.gdn_prefill_static.argtypes = [_P] * 10 + [_I] * 9 + [_F, _P, _P]
 _lib.gdn_prefill_static_workspace_bytes.restype = _Z
 _lib.gdn_prefill_static_workspace_bytes.argtypes = []
+_lib.gdn_decode_host_staging_bytes.restype = _Z
+_lib.gdn_decode_host_staging_bytes.argtypes = [_I] * 3
+_lib.gdn_decode_host.restype = ctypes.c_int
+_lib.gdn_decode_host.argtypes = [_P] * 8 + [_I] * 6 + [_F, _P, _Z, _P, _P]
+_lib.gdn_prefill_host_staging_bytes.restype = _Z
+_lib.gdn_prefill_host_staging_bytes.argtypes = [_I] * 4
+_lib.gdn_prefill_host.restype = ctypes.c_int
+_lib.gdn_prefill_host.argtypes = [_P] * 10 + [_I] * 9 + [_F, _P, _Z, _P, _Z, _P, _P]
 _lib.gdn_status_string.restype = ctypes.c_char_p
 _lib.gdn_status_string.argtypes = [ctypes.c_int]
 _lib.gdn_last_cuda_error_string.restype = ctypes.c_char_p
@@ -170,3 +179,59 @@ def gdn_prefill_static(q, k, v, g, beta, cu_seqlens, init_state, final_state, sl
         float(scale), _dev(dev_status, torch.int32, "dev_status", True), _stream())
     if rc != 0:
         raise GdnError(rc, "gdn_prefill_static")
+
+
+def _host(t, dtype, name, allow_none=False):
+    if t is None:
+        if allow_none:
+            return None
+        raise TypeError(f"{name} is required")
+    if not (isinstance(t, torch.Tensor) and not t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError(f"{name} must be a contiguous host tensor of dtype {dtype}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def gdn_decode_host_staging_bytes(B, Hqk, Hv) -> int:
+    return int(_lib.gdn_decode_host_staging_bytes(B, Hqk, Hv))
+
+
+def gdn_decode_host(q, k, v, g, beta, state_pool, slot_idx, o, scale, staging, dev_status=None):
+    """gdn_decode with host (pinned) q, k, v, g, beta, slot_idx and o; the state pool, the uint8
+    staging tensor and dev_status are CUDA tensors.  o is valid after a stream synchronise."""
+    B, Hqk, dk = q.shape
+    _, Hv, dv = v.shape
+    rc = _lib.gdn_decode_host(
+        _host(q, torch.bfloat16, "q"), _host(k, torch.bfloat16, "k"), _host(v, torch.bfloat16, "v"),
+        _host(g, torch.float32, "g"), _host(beta, torch.float32, "beta"),
+        _dev(state_pool, torch.float32, "state_pool"),
+        _host(slot_idx, torch.int32, "slot_idx", True), _host(o, torch.bfloat16, "o"),
+        B, Hqk, Hv, dk, dv, state_pool.shape[0], float(scale),
+        _dev(staging, torch.uint8, "staging"), staging.numel(),
+        _dev(dev_status, torch.int32, "dev_status", True), _stream())
+    if rc != 0:
+        raise GdnError(rc, "gdn_decode_host")
+
+
+def gdn_prefill_host_staging_bytes(T, N, Hqk, Hv) -> int:
+    return int(_lib.gdn_prefill_host_staging_bytes(T, N, Hqk, Hv))
+
+
+def gdn_prefill_host(q, k, v, g, beta, cu_seqlens, init_state, final_state, slot_idx, o, scale,
+                     staging, workspace, max_seqlen_hint=0, chunk=64, dev_status=None):
+    """gdn_prefill with host (pinned) q, k, v, g, beta, cu_seqlens, slot_idx and o."""
+    T, Hqk, dk = q.shape
+    _, Hv, dv = v.shape
+    N = cu_seqlens.shape[0] - 1
+    rc = _lib.gdn_prefill_host(
+        _host(q, torch.bfloat16, "q"), _host(k, torch.bfloat16, "k"), _host(v, torch.bfloat16, "v"),
+        _host(g, torch.float32, "g"), _host(beta, torch.float32, "beta"),
+        _host(cu_seqlens, torch.int32, "cu_seqlens"),
+        _dev(init_state, torch.float32, "init_state", True),
+        _dev(final_state, torch.float32, "final_state"),
+        _host(slot_idx, torch.int32, "slot_idx", True), _host(o, torch.bfloat16, "o"),
+        T, N, int(max_seqlen_hint), Hqk, Hv, dk, dv, int(chunk), final_state.shape[0],
+        float(scale), _dev(staging, torch.uint8, "staging"), staging.numel(),
+        _dev(workspace, torch.uint8, "workspace"), workspace.numel(),
+        _dev(dev_status, torch.int32, "dev_status", True), _stream())
+    if rc != 0:
+        raise GdnError(rc, "gdn_prefill_host")

@@ -192,6 +192,116 @@ int gdn_prefill(const void* q, const void* k, const void* v, const float* g, con
                                 scale, workspace, workspace_bytes, dev_status, stream);
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Host-buffer variants: per-call tensors live in (preferably pinned) host memory; they are copied
+// into a caller-provided device staging buffer, the device entry point runs, and o is copied
+// back, all enqueued on `stream`.
+// ---------------------------------------------------------------------------------------------
+namespace {
+struct Staging {
+    size_t q, k, v, g, beta, idx, o, total;
+};
+inline size_t up256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
+Staging staging_layout(int64_t rows, int32_t Hqk, int32_t Hv, int64_t n_idx) {
+    Staging s;
+    size_t off = 0;
+    s.q = off; off += up256(static_cast<size_t>(rows) * Hqk * gdn::kD * 2);
+    s.k = off; off += up256(static_cast<size_t>(rows) * Hqk * gdn::kD * 2);
+    s.v = off; off += up256(static_cast<size_t>(rows) * Hv * gdn::kD * 2);
+    s.g = off; off += up256(static_cast<size_t>(rows) * Hv * 4);
+    s.beta = off; off += up256(static_cast<size_t>(rows) * Hv * 4);
+    s.idx = off; off += up256(static_cast<size_t>(n_idx) * 4);
+    s.o = off; off += up256(static_cast<size_t>(rows) * Hv * gdn::kD * 2);
+    s.total = off;
+    return s;
+}
+}  // namespace
+
+size_t gdn_decode_host_staging_bytes(int32_t B, int32_t Hqk, int32_t Hv) {
+    if (B < 0 || Hqk <= 0 || Hv <= 0) return 0;
+    return staging_layout(B, Hqk, Hv, B).total;
+}
+
+int gdn_decode_host(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                    float* state_pool, const int32_t* slot_idx, void* o,
+                    int32_t B, int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv, int32_t num_slots,
+                    float scale, void* staging, size_t staging_bytes, int32_t* dev_status,
+                    void* stream) {
+    if (B < 0) return GDN_ERR_SIZE;
+    const int rc = check_heads(Hqk, Hv, dk, dv);
+    if (rc != GDN_OK) return rc;
+    if (B == 0) return GDN_OK;
+    if (!q || !k || !v || !g || !beta || !state_pool || !o || !staging) return GDN_ERR_NULL;
+    if (misaligned(staging, 256)) return GDN_ERR_ALIGN;
+    const Staging s = staging_layout(B, Hqk, Hv, B);
+    if (staging_bytes < s.total) return GDN_ERR_WORKSPACE;
+    uint8_t* d = static_cast<uint8_t*>(staging);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t qk = static_cast<size_t>(B) * Hqk * gdn::kD * 2, vo = static_cast<size_t>(B) * Hv * gdn::kD * 2;
+    const size_t sc = static_cast<size_t>(B) * Hv * 4;
+    cudaError_t e = cudaMemcpyAsync(d + s.q, q, qk, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d + s.k, k, qk, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d + s.v, v, vo, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d + s.g, g, sc, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d + s.beta, beta, sc, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && slot_idx)
+        e = cudaMemcpyAsync(d + s.idx, slot_idx, static_cast<size_t>(B) * 4, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_status(e);
+    const int r = gdn_decode(d + s.q, d + s.k, d + s.v, reinterpret_cast<const float*>(d + s.g),
+                             reinterpret_cast<const float*>(d + s.beta), state_pool,
+                             slot_idx ? reinterpret_cast<const int32_t*>(d + s.idx) : nullptr,
+                             d + s.o, B, Hqk, Hv, dk, dv, num_slots, scale, dev_status, stream);
+    if (r != GDN_OK) return r;
+    return cuda_status(cudaMemcpyAsync(o, d + s.o, vo, cudaMemcpyDeviceToHost, st));
+}
+
+size_t gdn_prefill_host_staging_bytes(int32_t T, int32_t N, int32_t Hqk, int32_t Hv) {
+    if (T < 0 || N < 0 || Hqk <= 0 || Hv <= 0) return 0;
+    return staging_layout(T, Hqk, Hv, 2 * static_cast<int64_t>(N) + 1).total;
+}
+
+int gdn_prefill_host(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                     const int32_t* cu_seqlens, const float* init_state, float* final_state,
+                     const int32_t* slot_idx, void* o, int32_t T, int32_t N,
+                     int32_t max_seqlen_hint, int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv,
+                     int32_t chunk, int32_t num_slots, float scale, void* staging,
+                     size_t staging_bytes, void* workspace, size_t workspace_bytes,
+                     int32_t* dev_status, void* stream) {
+    if (T < 0 || N < 0) return GDN_ERR_SIZE;
+    const int rc = check_heads(Hqk, Hv, dk, dv);
+    if (rc != GDN_OK) return rc;
+    if (T == 0 || N == 0) return GDN_OK;
+    if (!q || !k || !v || !g || !beta || !cu_seqlens || !final_state || !o || !staging)
+        return GDN_ERR_NULL;
+    if (misaligned(staging, 256)) return GDN_ERR_ALIGN;
+    const Staging s = staging_layout(T, Hqk, Hv, 2 * static_cast<int64_t>(N) + 1);
+    if (staging_bytes < s.total) return GDN_ERR_WORKSPACE;
+    uint8_t* d = static_cast<uint8_t*>(staging);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t qk = static_cast<size_t>(T) * Hqk * gdn::kD * 2, vo = static_cast<size_t>(T) * Hv * gdn::kD * 2;
+    const size_t sc = static_cast<size_t>(T) * Hv * 4;
+    int32_t* d_cu = reinterpret_cast<int32_t*>(d + s.idx);
+    int32_t* d_slot = d_cu + (N + 1);
+    cudaError_t e = cudaMemcpyAsync(d + s.q, q, qk, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d + s.k, k, qk, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d + s.v, v, vo, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d + s.g, g, sc, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d + s.beta, beta, sc, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(d_cu, cu_seqlens, static_cast<size_t>(N + 1) * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && slot_idx)
+        e = cudaMemcpyAsync(d_slot, slot_idx, static_cast<size_t>(N) * 4, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_status(e);
+    const int r = gdn_prefill(d + s.q, d + s.k, d + s.v, reinterpret_cast<const float*>(d + s.g),
+                              reinterpret_cast<const float*>(d + s.beta), d_cu, init_state,
+                              final_state, slot_idx ? d_slot : nullptr, d + s.o, T, N,
+                              max_seqlen_hint, Hqk, Hv, dk, dv, chunk, num_slots, scale, workspace,
+                              workspace_bytes, dev_status, stream);
+    if (r != GDN_OK) return r;
+    return cuda_status(cudaMemcpyAsync(o, d + s.o, vo, cudaMemcpyDeviceToHost, st));
+}
+
 const char* gdn_status_string(int code) {
     switch (code) {
         case GDN_OK: return "ok";

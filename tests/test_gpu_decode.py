@@ -137,3 +137,43 @@ def test_decode_paged_pool_config_full_size():
     U.check_o(U.host_f64_from_bf16(o), o_ref, U.O_REL_L2_DECODE)
     got = pool[torch.from_numpy(idx.astype(np.int64)).cuda()].cpu().numpy().astype(np.float64)
     U.check_state(got, gathered, U.STATE_REL_L2_DECODE)
+
+
+def test_host_buffer_entry_points_match_device_entry_points():
+    """gdn_decode_host / gdn_prefill_host (pinned host tensors in, o back to the host) give the
+    same bits as the device-pointer entry points."""
+    from paper_2607_17979_b200 import api
+    d = I.decode_inputs(5, 2, 4, 128, 7, seed=77, slots="perm")
+    o_dev, pool_dev, _ = run_decode(d)
+    pin = lambda t: t.cpu().pin_memory()
+    pool = U.dev(d["state"])
+    h_o = torch.empty((5, 4, 128), dtype=torch.bfloat16).pin_memory()
+    staging = torch.empty(api.gdn_decode_host_staging_bytes(5, 2, 4), dtype=torch.uint8, device="cuda")
+    api.gdn_decode_host(pin(U.dev_bf16(d["q"])), pin(U.dev_bf16(d["k"])), pin(U.dev_bf16(d["v"])),
+                        pin(U.dev(d["g"])), pin(U.dev(d["beta"])), pool, pin(U.dev(d["slot_idx"])),
+                        h_o, d["scale"], staging)
+    torch.cuda.synchronize()
+    assert np.array_equal(U.host_f64_from_bf16(h_o), o_dev)
+    assert np.array_equal(pool.cpu().numpy(), pool_dev)
+
+    p = I.prefill_inputs([100, 37], 2, 4, seed=78, init="normal")
+    T, N = p["T"], p["N"]
+    def run(host):
+        final = torch.empty((N, 4, 128, 128), dtype=torch.float32, device="cuda")
+        ws = torch.empty(api.gdn_prefill_workspace_bytes(T, N, 2, 4), dtype=torch.uint8, device="cuda")
+        dv = dict(q=U.dev_bf16(p["q"]), k=U.dev_bf16(p["k"]), v=U.dev_bf16(p["v"]), g=U.dev(p["g"]),
+                  beta=U.dev(p["beta"]), cu=U.dev(p["cu_seqlens"]))
+        if host:
+            o = torch.empty((T, 4, 128), dtype=torch.bfloat16).pin_memory()
+            st = torch.empty(api.gdn_prefill_host_staging_bytes(T, N, 2, 4), dtype=torch.uint8, device="cuda")
+            api.gdn_prefill_host(pin(dv["q"]), pin(dv["k"]), pin(dv["v"]), pin(dv["g"]), pin(dv["beta"]),
+                                 pin(dv["cu"]), U.dev(p["init_state"]), final, None, o, p["scale"], st, ws)
+        else:
+            o = torch.empty((T, 4, 128), dtype=torch.bfloat16, device="cuda")
+            api.gdn_prefill(dv["q"], dv["k"], dv["v"], dv["g"], dv["beta"], dv["cu"],
+                            U.dev(p["init_state"]), final, None, o, p["scale"], ws)
+        torch.cuda.synchronize()
+        return U.host_f64_from_bf16(o), final.cpu().numpy()
+    o_h, S_h = run(True)
+    o_d, S_d = run(False)
+    assert np.array_equal(o_h, o_d) and np.array_equal(S_h, S_d)
