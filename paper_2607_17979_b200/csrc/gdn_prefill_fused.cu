@@ -120,10 +120,10 @@ prefill_fused_prep_kernel(const int32_t* __restrict__ cu, int32_t T, int32_t N, 
 constexpr int kFusedThreads = 768;
 constexpr int kFGroups = 3;                          // intra role: three groups of 256 threads
 constexpr uint32_t kFGroupSmem = (kI_End + 1023u) & ~1023u;
-constexpr int kFEpiWarps = 16;                       // state role: warps 0-15 chain, warp 16 issues
+constexpr int kFEpiWarps = 8;                        // state role: warps 0-7 chain
 constexpr int kFEpiThreads = kFEpiWarps * 32;
-constexpr int kFIssueWarp = kFEpiWarps;              //   warp 16: tcgen05.mma issue
-constexpr int kFLoadWarp = kFEpiWarps + 1;           //   warp 17: record flags and TMA copies
+constexpr int kFIssueWarp = kFEpiWarps;              //   warp 8: tcgen05.mma issue
+constexpr int kFLoadWarp = kFEpiWarps + 1;           //   warp 9: record flags and TMA copies
 constexpr int kFRoleThreads = kFEpiThreads + 64;     // threads that take part in the state role
 constexpr uint32_t kFStateSmem = 2 * kStageBytes + 16384;
 constexpr uint32_t kFusedSmem =
@@ -210,7 +210,7 @@ __device__ __forceinline__ void fused_state_role(const TensorMaps& maps, const P
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (warp > kFLoadWarp) return;                    // spare warps of the CTA
     const bool is_epi = warp < kFEpiWarps;
-    const int part = warp >> 2;                       // which quarter of the columns this thread owns
+    const int half = (warp >> 2) & 1;                 // which half of the columns this thread owns
     const int dv = (warp & 3) * 32 + lane;            // TMEM lane = state row
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
     int32_t* hdr = reinterpret_cast<int32_t*>(ws);
@@ -273,11 +273,11 @@ __device__ __forceinline__ void fused_state_role(const TensorMaps& maps, const P
             continue;
         }
         const size_t tile_off = (static_cast<size_t>(slot) * p.Hv + hv) * (kD * kD) +
-                                static_cast<size_t>(dv) * kD + part * 32;
+                                static_cast<size_t>(dv) * kD + half * 64;
         if (nc == 0) {          // empty sequence: the state passes through untouched
             if (is_epi) {
-#pragma unroll
-                for (int j = 0; j < 32; j += 4) {
+#pragma unroll 4
+                for (int j = 0; j < 64; j += 4) {
                     const float4 x = p.init_state
                                          ? *reinterpret_cast<const float4*>(p.init_state + tile_off + j)
                                          : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -375,8 +375,9 @@ __device__ __forceinline__ void fused_state_role(const TensorMaps& maps, const P
                     mma_ts_c<true>(tY, tS + 56, sdesc_advance(qg, 8192 + 96), id64);
                     if (!wait_or_abort(&ss.bar_u, par_chunk(j), abortp)) break;    // U operands in TMEM
                     tc_fence_after_sync();
-                    // D4 = (U decayed, hi + lo) K   (K tile MN-major: 16 tokens = 2048 bytes)
-                    mma_ts_c<false>(tD4, tmem + kT_Us, kk, id128mn);
+                    // S_acc (= e^{b_C} S, prepared by the epilogue) += (U decayed, hi + lo) K
+                    // (K tile MN-major: 16 tokens = 2048 bytes)
+                    mma_ts_c<true>(tD4, tmem + kT_Us, kk, id128mn);
                     mma_ts_c<true>(tD4, tmem + kT_Us + 8, sdesc_advance(kk, 2048), id128mn);
                     mma_ts_c<true>(tD4, tmem + kT_Us + 16, sdesc_advance(kk, 4096), id128mn);
                     mma_ts_c<true>(tD4, tmem + kT_Us + 24, sdesc_advance(kk, 6144), id128mn);
@@ -396,42 +397,43 @@ __device__ __forceinline__ void fused_state_role(const TensorMaps& maps, const P
             }
             __syncwarp();
         } else {
-            // ===================== epilogue warps: the fp32 state and U (the dependent chain)
+            // ===================== epilogue warps: U and the state refresh (the dependent chain)
+            // The fp32 master state lives in TMEM (tile kT_D4): before chunk j's state product it
+            // holds e^{b_C(j)} S(j), the product accumulates U^T K into it, and the refresh below
+            // turns the result S(j+1) into the bf16 operand copy and into e^{b_C(j+1)} S(j+1).
             auto hand_over = [&](uint64_t* bar) {     // after tcgen05.st: publish to the issuing lane
                 tmem_wait_st();
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar);
             };
-            // the thread's 32 state columns [32*part, 32*part+32) of row dv, fp32 master copy
-            float S[32];
-            if (p.init_state) {
+            const uint32_t tSacc = tmem + kT_D4 + lane_base + half * 64;     // this thread's 64 columns
+            const uint32_t tSbf = tmem + kT_S + lane_base + half * 32;
+            // 16 state columns at a time: fp32 values v[] -> bf16 copy, and gamma * v -> master
+            auto put_state = [&](const int c0, const float (&v)[16], const float gamma) {
+                uint32_t pk[8], sc[16];
 #pragma unroll
-                for (int j = 0; j < 32; j += 4) {
-                    const float4 x = *reinterpret_cast<const float4*>(p.init_state + tile_off + j);
-                    S[j] = x.x; S[j + 1] = x.y; S[j + 2] = x.z; S[j + 3] = x.w;
-                }
-            } else {
+                for (int i = 0; i < 8; ++i) pk[i] = pack_bf16(v[2 * i], v[2 * i + 1]);
 #pragma unroll
-                for (int j = 0; j < 32; ++j) S[j] = 0.f;
-            }
-            auto store_state_bf16 = [&]() {           // S (fp32 regs) -> bf16 A operand in TMEM
-                uint32_t pk[16];
-#pragma unroll
-                for (int j = 0; j < 16; ++j) pk[j] = pack_bf16(S[2 * j], S[2 * j + 1]);
-                tmem_st16(tmem + kT_S + lane_base + part * 16, pk);
+                for (int i = 0; i < 16; ++i) sc[i] = __float_as_uint(gamma * v[i]);
+                tmem_st8(tSbf + (c0 >> 1), pk);
+                tmem_st16(tSacc + c0, sc);
             };
             // o rows of chunk j from Y[j & 1] in two parts that fit the two waits of the chain:
             // (A) scale, round, transpose into shared memory; (B) whole rows in 16-byte pieces
             auto outputs_stage = [&](int j) {
                 const uint32_t tY = tmem + kT_Y + (j & 1) * 64;
                 __nv_bfloat16* sO = reinterpret_cast<__nv_bfloat16*>(smem + kS_Out);
-                uint32_t x[16];
-                tmem_ld16(tY + lane_base + part * 16, x);
-                tmem_wait_ld();
 #pragma unroll
-                for (int jj = 0; jj < 16; ++jj)
-                    sO[(part * 16 + jj) * kD + dv] = __float2bfloat16(p.scale * __uint_as_float(x[jj]));
+                for (int c0 = 0; c0 < 32; c0 += 16) {
+                    uint32_t x[16];
+                    tmem_ld16(tY + lane_base + half * 32 + c0, x);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int jj = 0; jj < 16; ++jj)
+                        sO[(half * 32 + c0 + jj) * kD + dv] =
+                            __float2bfloat16(p.scale * __uint_as_float(x[jj]));
+                }
             };
             auto outputs_flush = [&](int j) {
                 const __nv_bfloat16* sO = reinterpret_cast<const __nv_bfloat16*>(smem + kS_Out);
@@ -439,27 +441,42 @@ __device__ __forceinline__ void fused_state_role(const TensorMaps& maps, const P
                 __nv_bfloat16* og = p.o + (static_cast<size_t>(seq_t0 + j * kChunk) * p.Hv + hv) * kD;
                 const size_t tok_stride = static_cast<size_t>(p.Hv) * kD;
 #pragma unroll
-                for (int it = 0; it < 2; ++it) {
-                    const int row = it * 32 + (tid >> 4), piece = tid & 15;
+                for (int it = 0; it < 4; ++it) {
+                    const int row = it * 16 + (tid >> 4), piece = tid & 15;
                     if (row < len)
                         *reinterpret_cast<uint4*>(og + row * tok_stride + piece * 8) =
                             *reinterpret_cast<const uint4*>(sO + row * kD + piece * 8);
                 }
             };
 
-            store_state_bf16();
-            hand_over(&ss.bar_s);
             bool ok = true;
             auto await = [&](uint64_t* bar, uint32_t parity) {   // bounded wait + tcgen05 fence
                 if (ok && !warp_wait_or_abort(bar, parity, abortp)) ok = false;
                 tc_fence_after_sync();
             };
+            // Every warp runs every group barrier and hand-over below, also after a wait has
+            // failed (ok == false: later waits and all work are skipped), so that no warp is ever
+            // left alone at a barrier.
+            await(&ss.bar_full[0], par_full(0));          // chunk 0's record: its e^{b_C} is needed
+            if (ok) {
+                const float g0 = reinterpret_cast<const float*>(smem + kS_Rec + kRecGammaC)[0];
+#pragma unroll 1
+                for (int c0 = 0; c0 < 64; c0 += 16) {
+                    float v[16];
+#pragma unroll
+                    for (int i = 0; i < 16; i += 4) {
+                        const float4 x = p.init_state
+                                             ? *reinterpret_cast<const float4*>(p.init_state + tile_off + c0 + i)
+                                             : make_float4(0.f, 0.f, 0.f, 0.f);
+                        v[i] = x.x; v[i + 1] = x.y; v[i + 2] = x.z; v[i + 3] = x.w;
+                    }
+                    put_state(c0, v, g0);
+                }
+            }
+            hand_over(&ss.bar_s);
             for (int j = 0; j < nc; ++j) {
                 const int st = j & 1;
                 const uint8_t* base = smem + st * kStageBytes;
-                // Every warp runs every group barrier and hand-over of every iteration, also after a
-                // wait has failed (ok == false: later waits and all work are skipped), so that no
-                // warp is ever left alone at a barrier.
                 if (j > 0) {     // part A of the previous chunk's outputs, while D1 is in flight
                     await(&ss.bar_y, par_chunk(j - 1));
                     epi_sync();
@@ -467,54 +484,68 @@ __device__ __forceinline__ void fused_state_role(const TensorMaps& maps, const P
                 }
                 await(&ss.bar_full[st], par_full(j));
                 await(&ss.bar_d1, par_chunk(j));
-                if (ok) {   // U^T[dv][c] = U~^T - D1 for the thread's 16 tokens [16*part, 16*part+16)
+                if (ok) {   // U^T[dv][c] = U~^T - D1 for the thread's 32 tokens [32*half, 32*half+32)
                     const float4* sU = reinterpret_cast<const float4*>(base + kS_Rec + kRecU);
                     const float* sdec = reinterpret_cast<const float*>(base + kS_Rec + kRecDecay);
-                    const int cb = part * 16;
-                    uint32_t x[16];
-                    tmem_ld16(tmem + kT_D1 + lane_base + cb, x);
-                    tmem_wait_ld();
-                    uint32_t pu[8], ph[8], pl[8];
 #pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        const float4 ut = sU[((cb >> 2) + q4) * kD + dv];
-                        const float4 dd = *reinterpret_cast<const float4*>(sdec + cb + 4 * q4);
-                        const float u0 = ut.x - __uint_as_float(x[4 * q4 + 0]);
-                        const float u1 = ut.y - __uint_as_float(x[4 * q4 + 1]);
-                        const float u2 = ut.z - __uint_as_float(x[4 * q4 + 2]);
-                        const float u3 = ut.w - __uint_as_float(x[4 * q4 + 3]);
-                        const float s0 = u0 * dd.x, s1 = u1 * dd.y, s2 = u2 * dd.z, s3 = u3 * dd.w;
-                        pu[2 * q4] = pack_bf16(u0, u1);
-                        pu[2 * q4 + 1] = pack_bf16(u2, u3);
-                        ph[2 * q4] = pack_bf16(s0, s1);
-                        ph[2 * q4 + 1] = pack_bf16(s2, s3);
-                        pl[2 * q4] = pack_bf16(s0 - __uint_as_float(ph[2 * q4] << 16),
-                                               s1 - __uint_as_float(ph[2 * q4] & 0xffff0000u));
-                        pl[2 * q4 + 1] = pack_bf16(s2 - __uint_as_float(ph[2 * q4 + 1] << 16),
-                                                   s3 - __uint_as_float(ph[2 * q4 + 1] & 0xffff0000u));
+                    for (int c0 = 0; c0 < 32; c0 += 16) {
+                        const int cb = half * 32 + c0;
+                        uint32_t x[16];
+                        tmem_ld16(tmem + kT_D1 + lane_base + cb, x);
+                        tmem_wait_ld();
+                        uint32_t pu[8], ph[8], pl[8];
+#pragma unroll
+                        for (int q4 = 0; q4 < 4; ++q4) {
+                            const float4 ut = sU[((cb >> 2) + q4) * kD + dv];
+                            const float4 dd = *reinterpret_cast<const float4*>(sdec + cb + 4 * q4);
+                            const float u0 = ut.x - __uint_as_float(x[4 * q4 + 0]);
+                            const float u1 = ut.y - __uint_as_float(x[4 * q4 + 1]);
+                            const float u2 = ut.z - __uint_as_float(x[4 * q4 + 2]);
+                            const float u3 = ut.w - __uint_as_float(x[4 * q4 + 3]);
+                            const float s0 = u0 * dd.x, s1 = u1 * dd.y, s2 = u2 * dd.z, s3 = u3 * dd.w;
+                            pu[2 * q4] = pack_bf16(u0, u1);
+                            pu[2 * q4 + 1] = pack_bf16(u2, u3);
+                            ph[2 * q4] = pack_bf16(s0, s1);
+                            ph[2 * q4 + 1] = pack_bf16(s2, s3);
+                            pl[2 * q4] = pack_bf16(s0 - __uint_as_float(ph[2 * q4] << 16),
+                                                   s1 - __uint_as_float(ph[2 * q4] & 0xffff0000u));
+                            pl[2 * q4 + 1] = pack_bf16(s2 - __uint_as_float(ph[2 * q4 + 1] << 16),
+                                                       s3 - __uint_as_float(ph[2 * q4 + 1] & 0xffff0000u));
+                        }
+                        tmem_st8(tmem + kT_Us + lane_base + (cb >> 1), ph);
+                        tmem_st8(tmem + kT_UsLo + lane_base + (cb >> 1), pl);
+                        tmem_st8(tmem + kT_U + lane_base + (cb >> 1), pu);
                     }
-                    tmem_st8(tmem + kT_Us + lane_base + (cb >> 1), ph);
-                    tmem_st8(tmem + kT_UsLo + lane_base + (cb >> 1), pl);
-                    tmem_st8(tmem + kT_U + lane_base + (cb >> 1), pu);
                 }
                 hand_over(&ss.bar_u);
                 if (j > 0) {     // part B, while this chunk's state product is in flight
                     epi_sync();
                     if (ok) outputs_flush(j - 1);
                 }
+                const bool last = j + 1 == nc;
+                if (!last) await(&ss.bar_full[st ^ 1], par_full(j + 1));   // next record's e^{b_C}
                 await(&ss.bar_d4, par_chunk(j));
-                if (ok) {   // S <- e^{b_C} S + D4 on the thread's 32 dk columns; refresh the bf16 copy
-                    const float gC = reinterpret_cast<const float*>(base + kS_Rec + kRecGammaC)[0];
-                    uint32_t xa[16], xb[16];
-                    tmem_ld16(tmem + kT_D4 + lane_base + part * 32, xa);
-                    tmem_ld16(tmem + kT_D4 + lane_base + part * 32 + 16, xb);
-                    tmem_wait_ld();
+                if (ok) {   // the master now holds S(j+1): refresh the bf16 copy, pre-scale the master
+                    const float gn = last ? 1.f
+                                          : reinterpret_cast<const float*>(smem + (st ^ 1) * kStageBytes +
+                                                                           kS_Rec + kRecGammaC)[0];
+#pragma unroll 2
+                    for (int c0 = 0; c0 < 64; c0 += 16) {
+                        uint32_t x[16];
+                        tmem_ld16(tSacc + c0, x);
+                        tmem_wait_ld();
+                        float v[16];
 #pragma unroll
-                    for (int jj = 0; jj < 16; ++jj) {
-                        S[jj] = fmaf(gC, S[jj], __uint_as_float(xa[jj]));
-                        S[16 + jj] = fmaf(gC, S[16 + jj], __uint_as_float(xb[jj]));
+                        for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(x[i]);
+                        if (!last) {
+                            put_state(c0, v, gn);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 16; i += 4)
+                                *reinterpret_cast<float4*>(p.final_state + tile_off + c0 + i) =
+                                    make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                        }
                     }
-                    store_state_bf16();
                 }
                 if (lane == 0) mbar_arrive(&ss.bar_free[st]);     // this warp is done with the stage
                 hand_over(&ss.bar_s);
@@ -524,12 +555,6 @@ __device__ __forceinline__ void fused_state_role(const TensorMaps& maps, const P
             if (ok) outputs_stage(nc - 1);
             epi_sync();
             if (ok) outputs_flush(nc - 1);
-            if (ok && !*abortp) {
-#pragma unroll
-                for (int j = 0; j < 32; j += 4)
-                    *reinterpret_cast<float4*>(p.final_state + tile_off + j) =
-                        make_float4(S[j], S[j + 1], S[j + 2], S[j + 3]);
-            }
         }
         tc_fence_before_sync();
         role_sync();                                   // end of the unit: barriers are re-armed next
