@@ -83,6 +83,36 @@ int gdn_decode(const void* q, const void* k, const void* v,
                int32_t* dev_status, void* stream);
 
 /*
+ * gdn_decode_multi - L >= 1 new tokens of the gated delta rule for each of B
+ * sequences in one call, applied in order, with a choice of state orientation
+ * (paper, same subsection: decode "computes a small number of new recurrent
+ * updates"; the paper's decode routes differ in "state layout", one of them
+ * working on the transposed tile).  The result equals L successive gdn_decode
+ * calls; the state tile is read and written once for all L tokens.
+ *
+ *   q, k        bf16 [B][L][Hqk][dk]
+ *   v           bf16 [B][L][Hv][dv]
+ *   g, beta     fp32 [B][L][Hv]
+ *   state_pool  fp32, updated in place:
+ *                 state_layout == GDN_STATE_VK: [num_slots][Hv][dv][dk] (as gdn_decode)
+ *                 state_layout == GDN_STATE_KV: [num_slots][Hv][dk][dv] (the transposed tile)
+ *   slot_idx    int32 [B] or NULL, rules as in gdn_decode (a padding entry's
+ *               L o rows are zero)
+ *   o           bf16 [B][L][Hv][dv], written
+ * L > GDN_DECODE_MAX_TOKENS returns GDN_ERR_LIMIT; another state_layout value
+ * returns GDN_ERR_SHAPE; B == 0 or L == 0 is a no-op that returns 0.
+ */
+#define GDN_DECODE_MAX_TOKENS 16
+#define GDN_STATE_VK 0
+#define GDN_STATE_KV 1
+int gdn_decode_multi(const void* q, const void* k, const void* v,
+                     const float* g, const float* beta,
+                     float* state_pool, const int32_t* slot_idx, void* o,
+                     int32_t B, int32_t L, int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv,
+                     int32_t num_slots, float scale, int32_t state_layout,
+                     int32_t* dev_status, void* stream);
+
+/*
  * gdn_prefill_workspace_bytes - device scratch gdn_prefill needs for a packed
  * batch of at most T tokens in at most N sequences.  Returns 0 for shapes
  * gdn_prefill would reject.

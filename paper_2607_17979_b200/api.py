@@ -37,6 +37,8 @@ _P, _I, _F, _Z = ctypes.c_void_p, ctypes.c_int32, ctypes.c_float, ctypes.c_size_
 _lib.gdn_decode.restype = ctypes.c_int
 _lib.gdn_decode.argtypes = [_P] * 8 + [_I] * 6 + [_F, _P, _P]
 _lib.gdn_prefill_workspace_bytes.restype = _Z
+_lib.gdn_decode_multi.restype = ctypes.c_int
+_lib.gdn_decode_multi.argtypes = [_P] * 8 + [_I] * 7 + [_F, _I, _P, _P]
 _lib.gdn_prefill_workspace_bytes.argtypes = [_I] * 7
 _lib.gdn_prefill.restype = ctypes.c_int
 _lib.gdn_prefill.argtypes = [_P] * 10 + [_I] * 9 + [_F, _P, _Z, _P, _P]
@@ -106,6 +108,27 @@ def gdn_decode(q, k, v, g, beta, state_pool, slot_idx, o, scale, dev_status=None
         _dev(dev_status, torch.int32, "dev_status", True), _stream())
     if rc != 0:
         raise GdnError(rc, "gdn_decode")
+
+
+DECODE_MAX_TOKENS = 16
+STATE_VK, STATE_KV = 0, 1
+
+
+def gdn_decode_multi(q, k, v, g, beta, state_pool, slot_idx, o, scale, state_layout=STATE_VK,
+                     dev_status=None):
+    """L new tokens per sequence in one call (q [B,L,Hqk,128], v/o [B,L,Hv,128], g/beta [B,L,Hv]);
+    ``state_layout`` STATE_VK = tiles [dv][dk], STATE_KV = tiles [dk][dv]."""
+    B, L, Hqk, dk = q.shape
+    _, _, Hv, dv = v.shape
+    rc = _lib.gdn_decode_multi(
+        _dev(q, torch.bfloat16, "q"), _dev(k, torch.bfloat16, "k"), _dev(v, torch.bfloat16, "v"),
+        _dev(g, torch.float32, "g"), _dev(beta, torch.float32, "beta"),
+        _dev(state_pool, torch.float32, "state_pool"),
+        _dev(slot_idx, torch.int32, "slot_idx", True), _dev(o, torch.bfloat16, "o"),
+        B, L, Hqk, Hv, dk, dv, state_pool.shape[0], float(scale), int(state_layout),
+        _dev(dev_status, torch.int32, "dev_status", True), _stream())
+    if rc != 0:
+        raise GdnError(rc, "gdn_decode_multi")
 
 
 def gdn_prefill_workspace_bytes(T, N, Hqk, Hv, dk=128, dv=128, chunk=64) -> int:

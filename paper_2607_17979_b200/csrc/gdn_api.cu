@@ -70,6 +70,37 @@ int gdn_decode(const void* q, const void* k, const void* v, const float* g, cons
     return cuda_status(gdn::launch_decode(p, static_cast<cudaStream_t>(stream)));
 }
 
+int gdn_decode_multi(const void* q, const void* k, const void* v, const float* g,
+                     const float* beta, float* state_pool, const int32_t* slot_idx, void* o,
+                     int32_t B, int32_t L, int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv,
+                     int32_t num_slots, float scale, int32_t state_layout, int32_t* dev_status,
+                     void* stream) {
+    if (B < 0 || L < 0) return GDN_ERR_SIZE;
+    const int rc = check_heads(Hqk, Hv, dk, dv);
+    if (rc != GDN_OK) return rc;
+    if (state_layout != GDN_STATE_VK && state_layout != GDN_STATE_KV) return GDN_ERR_SHAPE;
+    if (L > GDN_DECODE_MAX_TOKENS) return GDN_ERR_LIMIT;
+    if (B == 0 || L == 0) return GDN_OK;
+    if (num_slots <= 0) return GDN_ERR_SIZE;
+    if (!q || !k || !v || !g || !beta || !state_pool || !o) return GDN_ERR_NULL;
+    if (misaligned(q, 16) || misaligned(k, 16) || misaligned(v, 16) || misaligned(o, 16) ||
+        misaligned(state_pool, 16) || misaligned(g, 4) || misaligned(beta, 4) ||
+        misaligned(slot_idx, 4) || misaligned(dev_status, 4))
+        return GDN_ERR_ALIGN;
+    gdn::DecodeMultiParams mp;
+    gdn::DecodeParams& p = mp.d;
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.k = static_cast<const __nv_bfloat16*>(k);
+    p.v = static_cast<const __nv_bfloat16*>(v);
+    p.g = g; p.beta = beta; p.pool = state_pool; p.slot_idx = slot_idx;
+    p.o = static_cast<__nv_bfloat16*>(o);
+    p.B = B; p.Hqk = Hqk; p.Hv = Hv; p.num_slots = num_slots; p.scale = scale;
+    p.dev_status = dev_status;
+    mp.L = L;
+    mp.layout = state_layout;
+    return cuda_status(gdn::launch_decode_multi(mp, static_cast<cudaStream_t>(stream)));
+}
+
 size_t gdn_prefill_workspace_bytes(int32_t T, int32_t N, int32_t Hqk, int32_t Hv,
                                    int32_t dk, int32_t dv, int32_t chunk) {
     if (T < 0 || N < 0 || chunk != gdn::kChunk || check_heads(Hqk, Hv, dk, dv) != GDN_OK) return 0;

@@ -9,6 +9,7 @@ namespace gdn {
 
 constexpr int kD = 128;          // dk == dv == 128 is the only supported head size
 constexpr int kChunk = 64;       // prefill chunk length
+constexpr int kDecodeMaxTokens = 16;  // most new tokens per sequence in one multi-token decode
 
 // device status bits (mirror GDN_DEV_* of the public header)
 constexpr int kDevBadSlot = 1;
@@ -29,6 +30,12 @@ struct DecodeParams {
     int32_t* dev_status;
 };
 
+struct DecodeMultiParams {
+    DecodeParams d;      // q,k [B][L][Hqk][128]; v,o [B][L][Hv][128]; g,beta [B][L][Hv]
+    int32_t L;           // new tokens per sequence, 1..kDecodeMaxTokens
+    int32_t layout;      // 0: tile [dv][dk];  1: tile [dk][dv]
+};
+
 struct PrefillParams {
     const __nv_bfloat16* q;
     const __nv_bfloat16* k;
@@ -46,6 +53,7 @@ struct PrefillParams {
 };
 
 cudaError_t launch_decode(const DecodeParams& p, cudaStream_t stream);
+cudaError_t launch_decode_multi(const DecodeMultiParams& mp, cudaStream_t stream);
 cudaError_t launch_prefill_recurrent(const PrefillParams& p, cudaStream_t stream);
 
 __device__ __forceinline__ void report(int32_t* dev_status, int bit) {

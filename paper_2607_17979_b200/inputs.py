@@ -103,6 +103,29 @@ def decode_inputs(B: int, Hqk: int, Hv: int, d: int = 128, num_slots: int | None
                 B=B, Hqk=Hqk, Hv=Hv, dk=d, dv=d, num_slots=num_slots)
 
 
+def decode_multi_inputs(B: int, L: int, Hqk: int, Hv: int, d: int = 128,
+                        num_slots: int | None = None, seed: int = BASE_SEED,
+                        alpha_lo: float = 0.9, slots: str = "identity",
+                        state: str = "normal") -> dict:
+    """Inputs of one multi-token decode call: L new tokens for each of B sequences
+    (q, k [B, L, Hqk, d]; v [B, L, Hv, d]; g, beta [B, L, Hv]); pool and slots as in
+    decode_inputs.  ``state`` holds tiles [dv][dk]."""
+    num_slots = B if num_slots is None else num_slots
+    q = _unit_vectors_bf16(rng(seed, "q"), (B, L, Hqk, d))
+    k = _unit_vectors_bf16(rng(seed, "k"), (B, L, Hqk, d))
+    v = _normal_bf16(rng(seed, "v"), (B, L, Hv, d))
+    g, beta = _gates(seed, (B, L, Hv), alpha_lo)
+    pool = _state(seed, (num_slots, Hv, d, d), state)
+    slot_idx = None
+    if slots == "perm":
+        slot_idx = rng(seed, "slots").permutation(num_slots)[:B].astype(np.int32)
+    elif slots != "identity":
+        raise ValueError(slots)
+    return dict(q=q, k=k, v=v, g=g, beta=beta, state=pool, slot_idx=slot_idx,
+                scale=float(np.float32(1.0 / np.sqrt(d))),
+                B=B, L=L, Hqk=Hqk, Hv=Hv, dk=d, dv=d, num_slots=num_slots)
+
+
 def prefill_inputs(seq_lens, Hqk: int, Hv: int, d: int = 128, seed: int = BASE_SEED,
                    alpha_lo: float = 0.9, init: str = "zero") -> dict:
     """A packed variable-length prefill batch.

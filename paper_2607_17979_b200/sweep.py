@@ -20,6 +20,7 @@ import torch
 from . import api, inputs as I
 
 DECODE_BATCHES = [1, 4, 8, 16, 32, 48, 64]
+MULTI_SHAPES = [(1, 2), (1, 8), (8, 4), (32, 4), (64, 1), (64, 2), (64, 4), (64, 8)]
 PREFILL_SHAPES = [[6], [12], [35], [100], [256], [512], [1024], [300, 700], [2855, 2854],
                   [410] * 20, [144] * 56 + [128]]
 
@@ -73,6 +74,17 @@ def main():
                    args.reps)
         rows.append({"op": "decode", "B": B, "Hqk": 16, "Hv": 32, "us": us,
                      "state_GBps": 2 * B * 32 * 65536 / us / 1e3})
+    # multi-token decode (L new tokens per sequence in one call), both state orientations
+    for B, L in MULTI_SHAPES:
+        d = I.decode_multi_inputs(B, L, 16, 32, 128, B, seed=I.BASE_SEED + 7 * B + L)
+        t = {n: _bf16(d[n]) for n in "qkv"}
+        g, beta, pool = _dev(d["g"]), _dev(d["beta"]), _dev(d["state"])
+        o = torch.empty((B, L, 32, 128), dtype=torch.bfloat16, device="cuda")
+        for layout, name in ((api.STATE_VK, "vk"), (api.STATE_KV, "kv")):
+            us = _time(lambda: api.gdn_decode_multi(t["q"], t["k"], t["v"], g, beta, pool, None, o,
+                                                    d["scale"], layout), args.reps)
+            rows.append({"op": "decode_multi", "B": B, "L": L, "layout": name, "us": us,
+                         "tokens_per_s": B * L / us * 1e6})
     for lens in PREFILL_SHAPES:
         p = I.prefill_inputs(lens, 16, 32, 128, seed=I.BASE_SEED + sum(lens), init="zero")
         t = {n: _bf16(p[n]) for n in "qkv"}
