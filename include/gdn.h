@@ -113,6 +113,43 @@ int gdn_decode_multi(const void* q, const void* k, const void* v,
                      int32_t* dev_status, void* stream);
 
 /*
+ * gdn_gate - the scalar gate / beta preprocessing in front of the recurrence
+ * (paper: the prefill route keeps a small fused helper that prepares the gate
+ * and beta inputs; the paper prints no formula for it).  Reading taken: the
+ * parametrisation of the published Gated DeltaNet layer,
+ *     g[t][h]    = -exp(A_log[h]) * softplus(a[t][h] + dt_bias[h])
+ *     beta[t][h] = sigmoid(b[t][h])
+ * so that g <= 0 (alpha = exp(g) in (0, 1]) and beta in (0, 1).
+ *
+ *   a, b        bf16 [T][Hv]   raw per-token projections
+ *   A_log       fp32 [Hv]      per-head log decay rate
+ *   dt_bias     fp32 [Hv]      per-head bias
+ *   g, beta     fp32 [T][Hv], written: the g and beta arguments of gdn_prefill /
+ *               gdn_decode (T = B for a decode step)
+ * T == 0 is a no-op that returns 0.
+ */
+int gdn_gate(const void* a, const void* b, const float* A_log, const float* dt_bias,
+             float* g, float* beta, int32_t T, int32_t Hv, void* stream);
+
+/*
+ * gdn_state_transpose - transpose, in place, the 128 x 128 state tiles of n
+ * entries (all Hv heads each): [dv][dk] becomes [dk][dv] and back.  It lets a
+ * pool kept in the GDN_STATE_KV orientation go through gdn_prefill (which
+ * reads and writes GDN_STATE_VK tiles): transpose the touched slots, prefill,
+ * transpose again.  (The paper names the transposed-state decode route but no
+ * such helper; this is this library's addition.)
+ *
+ *   state_pool  fp32 [num_slots][Hv][128][128], tiles transposed in place
+ *   slot_idx    int32 [n] or NULL (= slots 0..n-1); negative entries are
+ *               skipped, entries >= num_slots are skipped and set
+ *               GDN_DEV_BAD_SLOT; a slot listed twice is undefined
+ * n == 0 is a no-op that returns 0.
+ */
+int gdn_state_transpose(float* state_pool, const int32_t* slot_idx, int32_t n, int32_t Hv,
+                        int32_t dk, int32_t dv, int32_t num_slots,
+                        int32_t* dev_status, void* stream);
+
+/*
  * gdn_prefill_workspace_bytes - device scratch gdn_prefill needs for a packed
  * batch of at most T tokens in at most N sequences.  Returns 0 for shapes
  * gdn_prefill would reject.

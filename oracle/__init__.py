@@ -124,3 +124,20 @@ def prefill(q, k, v, g, beta, cu_seqlens, init_state=None, slot_idx=None, scale=
     if rc < 0:
         raise ValueError(f"gdn_oracle_prefill rejected its arguments ({rc})")
     return o, final_state, rc
+
+
+def gate(a_bits, b_bits, A_log, dt_bias):
+    """Gate / beta preprocessing in fp64 (the paper names the helper without a formula; this is
+    the published Gated DeltaNet parametrisation, the reading the library documents):
+    g = -exp(A_log) * softplus(a + dt_bias), beta = sigmoid(b).
+
+    a_bits, b_bits: uint16 bf16 patterns [T, Hv]; A_log, dt_bias: float [Hv].
+    Returns (g, beta) float64 [T, Hv].
+    """
+    a = (np.ascontiguousarray(a_bits, np.uint16).astype(np.uint32) << 16).view(np.float32)
+    b = (np.ascontiguousarray(b_bits, np.uint16).astype(np.uint32) << 16).view(np.float32)
+    x = a.astype(np.float64) + np.asarray(dt_bias, np.float64)[None, :]
+    softplus = np.maximum(x, 0.0) + np.log1p(np.exp(-np.abs(x)))
+    g = -np.exp(np.asarray(A_log, np.float64))[None, :] * softplus
+    beta = 1.0 / (1.0 + np.exp(-b.astype(np.float64)))
+    return g, beta

@@ -39,6 +39,10 @@ _lib.gdn_decode.argtypes = [_P] * 8 + [_I] * 6 + [_F, _P, _P]
 _lib.gdn_prefill_workspace_bytes.restype = _Z
 _lib.gdn_decode_multi.restype = ctypes.c_int
 _lib.gdn_decode_multi.argtypes = [_P] * 8 + [_I] * 7 + [_F, _I, _P, _P]
+_lib.gdn_gate.restype = ctypes.c_int
+_lib.gdn_gate.argtypes = [_P] * 6 + [_I, _I, _P]
+_lib.gdn_state_transpose.restype = ctypes.c_int
+_lib.gdn_state_transpose.argtypes = [_P, _P] + [_I] * 5 + [_P, _P]
 _lib.gdn_prefill_workspace_bytes.argtypes = [_I] * 7
 _lib.gdn_prefill.restype = ctypes.c_int
 _lib.gdn_prefill.argtypes = [_P] * 10 + [_I] * 9 + [_F, _P, _Z, _P, _P]
@@ -129,6 +133,30 @@ def gdn_decode_multi(q, k, v, g, beta, state_pool, slot_idx, o, scale, state_lay
         _dev(dev_status, torch.int32, "dev_status", True), _stream())
     if rc != 0:
         raise GdnError(rc, "gdn_decode_multi")
+
+
+def gdn_gate(a, b, A_log, dt_bias, g, beta):
+    """g = -exp(A_log) * softplus(a + dt_bias), beta = sigmoid(b); a, b bf16 [T, Hv]."""
+    T, Hv = a.shape
+    rc = _lib.gdn_gate(_dev(a, torch.bfloat16, "a"), _dev(b, torch.bfloat16, "b"),
+                       _dev(A_log, torch.float32, "A_log"), _dev(dt_bias, torch.float32, "dt_bias"),
+                       _dev(g, torch.float32, "g"), _dev(beta, torch.float32, "beta"), T, Hv,
+                       _stream())
+    if rc != 0:
+        raise GdnError(rc, "gdn_gate")
+
+
+def gdn_state_transpose(state_pool, slot_idx=None, n=None, dev_status=None):
+    """Transpose in place the tiles of ``n`` entries (default: every slot) of a
+    [num_slots, Hv, 128, 128] fp32 CUDA pool."""
+    num_slots, Hv, dv, dk = state_pool.shape
+    if n is None:
+        n = slot_idx.shape[0] if slot_idx is not None else num_slots
+    rc = _lib.gdn_state_transpose(
+        _dev(state_pool, torch.float32, "state_pool"), _dev(slot_idx, torch.int32, "slot_idx", True),
+        int(n), Hv, dk, dv, num_slots, _dev(dev_status, torch.int32, "dev_status", True), _stream())
+    if rc != 0:
+        raise GdnError(rc, "gdn_state_transpose")
 
 
 def gdn_prefill_workspace_bytes(T, N, Hqk, Hv, dk=128, dv=128, chunk=64) -> int:

@@ -101,6 +101,34 @@ int gdn_decode_multi(const void* q, const void* k, const void* v, const float* g
     return cuda_status(gdn::launch_decode_multi(mp, static_cast<cudaStream_t>(stream)));
 }
 
+int gdn_gate(const void* a, const void* b, const float* A_log, const float* dt_bias,
+             float* g, float* beta, int32_t T, int32_t Hv, void* stream) {
+    if (T < 0 || Hv < 0) return GDN_ERR_SIZE;
+    if (T == 0 || Hv == 0) return GDN_OK;
+    if (!a || !b || !A_log || !dt_bias || !g || !beta) return GDN_ERR_NULL;
+    if (misaligned(a, 2) || misaligned(b, 2) || misaligned(A_log, 4) || misaligned(dt_bias, 4) ||
+        misaligned(g, 4) || misaligned(beta, 4))
+        return GDN_ERR_ALIGN;
+    return cuda_status(gdn::launch_gate(static_cast<const __nv_bfloat16*>(a),
+                                        static_cast<const __nv_bfloat16*>(b), A_log, dt_bias, g,
+                                        beta, static_cast<long long>(T) * Hv, Hv,
+                                        static_cast<cudaStream_t>(stream)));
+}
+
+int gdn_state_transpose(float* state_pool, const int32_t* slot_idx, int32_t n, int32_t Hv,
+                        int32_t dk, int32_t dv, int32_t num_slots, int32_t* dev_status,
+                        void* stream) {
+    if (n < 0 || Hv < 0) return GDN_ERR_SIZE;
+    if (dk != gdn::kD || dv != gdn::kD) return GDN_ERR_SHAPE;
+    if (n == 0 || Hv == 0) return GDN_OK;
+    if (num_slots <= 0) return GDN_ERR_SIZE;
+    if (!state_pool) return GDN_ERR_NULL;
+    if (misaligned(state_pool, 16) || misaligned(slot_idx, 4) || misaligned(dev_status, 4))
+        return GDN_ERR_ALIGN;
+    return cuda_status(gdn::launch_state_transpose(state_pool, slot_idx, n, Hv, num_slots,
+                                                   dev_status, static_cast<cudaStream_t>(stream)));
+}
+
 size_t gdn_prefill_workspace_bytes(int32_t T, int32_t N, int32_t Hqk, int32_t Hv,
                                    int32_t dk, int32_t dv, int32_t chunk) {
     if (T < 0 || N < 0 || chunk != gdn::kChunk || check_heads(Hqk, Hv, dk, dv) != GDN_OK) return 0;

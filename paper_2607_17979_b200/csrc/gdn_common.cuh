@@ -54,6 +54,11 @@ struct PrefillParams {
 
 cudaError_t launch_decode(const DecodeParams& p, cudaStream_t stream);
 cudaError_t launch_decode_multi(const DecodeMultiParams& mp, cudaStream_t stream);
+cudaError_t launch_gate(const __nv_bfloat16* a, const __nv_bfloat16* b, const float* A_log,
+                        const float* dt_bias, float* g, float* beta, long long n, int Hv,
+                        cudaStream_t stream);
+cudaError_t launch_state_transpose(float* pool, const int32_t* slot_idx, int32_t n, int32_t Hv,
+                                   int32_t num_slots, int32_t* dev_status, cudaStream_t stream);
 cudaError_t launch_prefill_recurrent(const PrefillParams& p, cudaStream_t stream);
 
 __device__ __forceinline__ void report(int32_t* dev_status, int bit) {

@@ -311,3 +311,49 @@ cudaError_t launch_decode_multi(const DecodeMultiParams& mp, cudaStream_t stream
 }
 
 }  // namespace gdn
+
+// ---- in-place transpose of state tiles ([dv][dk] <-> [dk][dv]) ---------------------------------
+// One CTA per (entry, v-head) tile.  The 128x128 tile is walked as 4x4 blocks of 32x32; a block
+// pair (a, b) and (b, a) is read into two padded shared tiles and written back swapped and
+// transposed, so the tile never needs a second copy in memory.
+namespace gdn {
+
+__global__ void __launch_bounds__(256)
+state_transpose_kernel(float* pool, const int32_t* slot_idx, int32_t Hv, int32_t num_slots,
+                       int32_t* dev_status) {
+    __shared__ float ta[32][33], tb[32][33];
+    const int i = blockIdx.x / Hv, hv = blockIdx.x - i * Hv;
+    const int slot = slot_idx ? slot_idx[i] : i;
+    if (slot < 0 || slot >= num_slots) {
+        if (slot >= num_slots && threadIdx.x == 0) report(dev_status, kDevBadSlot);
+        return;
+    }
+    float* tile = pool + (static_cast<size_t>(slot) * Hv + hv) * (kD * kD);
+    const int c = threadIdx.x & 31, r0 = threadIdx.x >> 5;   // 8 rows per sweep
+    for (int a = 0; a < 4; ++a)
+        for (int b = a; b < 4; ++b) {
+#pragma unroll
+            for (int r = r0; r < 32; r += 8) {
+                ta[r][c] = tile[(a * 32 + r) * kD + b * 32 + c];
+                tb[r][c] = tile[(b * 32 + r) * kD + a * 32 + c];
+            }
+            __syncthreads();
+#pragma unroll
+            for (int r = r0; r < 32; r += 8) {
+                tile[(b * 32 + r) * kD + a * 32 + c] = ta[c][r];
+                if (a != b) tile[(a * 32 + r) * kD + b * 32 + c] = tb[c][r];
+            }
+            __syncthreads();
+        }
+}
+
+cudaError_t launch_state_transpose(float* pool, const int32_t* slot_idx, int32_t n, int32_t Hv,
+                                   int32_t num_slots, int32_t* dev_status, cudaStream_t stream) {
+    const long long units = static_cast<long long>(n) * Hv;
+    if (units == 0) return cudaSuccess;
+    state_transpose_kernel<<<static_cast<unsigned>(units), 256, 0, stream>>>(pool, slot_idx, Hv,
+                                                                             num_slots, dev_status);
+    return cudaGetLastError();
+}
+
+}  // namespace gdn

@@ -23,7 +23,8 @@ import numpy as np
 
 BASE_SEED = 20260717
 
-_TAGS = {"q": 1, "k": 2, "v": 3, "alpha": 4, "beta": 5, "state": 6, "slots": 7}
+_TAGS = {"q": 1, "k": 2, "v": 3, "alpha": 4, "beta": 5, "state": 6, "slots": 7,
+         "gate_a": 8, "gate_b": 9, "A_log": 10, "dt_bias": 11}
 
 
 def rng(seed: int, tag: str) -> np.random.Generator:
@@ -124,6 +125,16 @@ def decode_multi_inputs(B: int, L: int, Hqk: int, Hv: int, d: int = 128,
     return dict(q=q, k=k, v=v, g=g, beta=beta, state=pool, slot_idx=slot_idx,
                 scale=float(np.float32(1.0 / np.sqrt(d))),
                 B=B, L=L, Hqk=Hqk, Hv=Hv, dk=d, dv=d, num_slots=num_slots)
+
+
+def gate_inputs(T: int, Hv: int, seed: int = BASE_SEED) -> dict:
+    """Raw inputs of the gate helper: a, b ~ N(0,1) as bf16 bits [T, Hv]; A_log = ln U[1,16) and
+    dt_bias ~ N(0,1), fp32 [Hv]."""
+    a = _normal_bf16(rng(seed, "gate_a"), (T, Hv))
+    b = _normal_bf16(rng(seed, "gate_b"), (T, Hv))
+    A_log = np.log(rng(seed, "A_log").uniform(1.0, 16.0, size=Hv)).astype(np.float32)
+    dt_bias = rng(seed, "dt_bias").standard_normal(Hv).astype(np.float32)
+    return dict(a=a, b=b, A_log=A_log, dt_bias=dt_bias, T=T, Hv=Hv)
 
 
 def prefill_inputs(seq_lens, Hqk: int, Hv: int, d: int = 128, seed: int = BASE_SEED,

@@ -137,3 +137,47 @@ def test_decode_multi_rejects_bad_arguments():
                              torch.empty((2, 2, 2, 128), dtype=torch.bfloat16, device="cuda"),
                              d["scale"], 2)
     assert e.value.code == -3
+
+
+def test_state_transpose_in_place_and_prefill_into_a_transposed_pool():
+    """gdn_state_transpose is bit-exact, skips unlisted slots, and brackets gdn_prefill so that a
+    pool kept as [dk][dv] tiles can be prefilled and then decoded in that orientation."""
+    from paper_2607_17979_b200 import api
+    rng = np.random.default_rng(5)
+    pool_h = rng.standard_normal((6, 4, 128, 128)).astype(np.float32)
+    pool = U.dev(pool_h)
+    idx = np.array([4, -1, 1, 7], np.int32)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    api.gdn_state_transpose(pool, U.dev(idx), dev_status=status)
+    torch.cuda.synchronize()
+    want = pool_h.copy()
+    want[[4, 1]] = pool_h[[4, 1]].transpose(0, 1, 3, 2)
+    assert np.array_equal(pool.cpu().numpy(), want) and int(status.item()) == 1
+    api.gdn_state_transpose(pool)            # every slot
+    torch.cuda.synchronize()
+    want = want.transpose(0, 1, 3, 2)
+    assert np.array_equal(pool.cpu().numpy(), want)
+
+    # prefill into a [dk][dv] pool, then one multi-token decode in that orientation
+    p = I.prefill_inputs([70, 130], 2, 4, seed=91, init="normal")
+    T, N = p["T"], p["N"]
+    kv_pool = U.dev(np.ascontiguousarray(p["init_state"].transpose(0, 1, 3, 2)))
+    o = torch.empty((T, 4, 128), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(api.gdn_prefill_workspace_bytes(T, N, 2, 4), dtype=torch.uint8, device="cuda")
+    api.gdn_state_transpose(kv_pool)
+    api.gdn_prefill(U.dev_bf16(p["q"]), U.dev_bf16(p["k"]), U.dev_bf16(p["v"]), U.dev(p["g"]),
+                    U.dev(p["beta"]), U.dev(p["cu_seqlens"]), kv_pool, kv_pool, None, o, p["scale"], ws)
+    api.gdn_state_transpose(kv_pool)
+    d = I.decode_multi_inputs(N, 3, 2, 4, 128, N, seed=92)
+    o2 = torch.empty((N, 3, 4, 128), dtype=torch.bfloat16, device="cuda")
+    api.gdn_decode_multi(U.dev_bf16(d["q"]), U.dev_bf16(d["k"]), U.dev_bf16(d["v"]), U.dev(d["g"]),
+                         U.dev(d["beta"]), kv_pool, None, o2, d["scale"], KV)
+    torch.cuda.synchronize()
+    o_ref, S_ref, _ = oracle.prefill(p["q"], p["k"], p["v"], p["g"], p["beta"], p["cu_seqlens"],
+                                     p["init_state"].astype(np.float64), None, p["scale"])
+    U.check_o(U.host_f64_from_bf16(o), o_ref, U.O_REL_L2_PREFILL)
+    d["state"] = S_ref
+    o2_ref, S2_ref, _ = oracle_multi(d)
+    U.check_o(U.host_f64_from_bf16(o2), o2_ref, U.O_REL_L2_PREFILL)
+    got = kv_pool.cpu().numpy().transpose(0, 1, 3, 2).astype(np.float64)
+    U.check_state(got, S2_ref, U.STATE_REL_L2_PREFILL)
