@@ -231,6 +231,24 @@ int gdn_prefill_fused(const void* q, const void* k, const void* v,
                       int32_t* dev_status, void* stream);
 
 /*
+ * gdn_prefill_stream - the chunked algorithm in three launches whose state
+ * pass is a persistent kernel: one CTA per SM walks a list of (sequence,
+ * v-head) units and streams their chunks without draining its pipeline
+ * between units.  It is the route for batches with many more units than SMs
+ * (many short sequences).  Arguments, workspace and results are
+ * gdn_prefill_chunked's.
+ */
+int gdn_prefill_stream(const void* q, const void* k, const void* v,
+                       const float* g, const float* beta, const int32_t* cu_seqlens,
+                       const float* init_state, float* final_state, const int32_t* slot_idx,
+                       void* o,
+                       int32_t T, int32_t N, int32_t max_seqlen_hint,
+                       int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv, int32_t chunk,
+                       int32_t num_slots, float scale,
+                       void* workspace, size_t workspace_bytes,
+                       int32_t* dev_status, void* stream);
+
+/*
  * gdn_prefill_recurrent - the same operator and arguments as gdn_prefill,
  * evaluated token by token on the CUDA cores (no chunking, no workspace).  The
  * rows of a state tile evolve independently under the gated delta rule, so the

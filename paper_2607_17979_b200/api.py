@@ -16,7 +16,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libgdn_b200.so")
 
 EXPORTS = ("gdn_decode", "gdn_prefill_workspace_bytes", "gdn_prefill", "gdn_prefill_chunked",
-           "gdn_prefill_fused", "gdn_decode_host", "gdn_decode_host_staging_bytes",
+           "gdn_prefill_fused", "gdn_prefill_stream", "gdn_decode_multi", "gdn_gate",
+           "gdn_state_transpose", "gdn_decode_host", "gdn_decode_host_staging_bytes",
            "gdn_prefill_host", "gdn_prefill_host_staging_bytes",
            "gdn_prefill_recurrent",
            "gdn_prefill_static", "gdn_prefill_static_workspace_bytes", "gdn_status_string",
@@ -50,6 +51,8 @@ _lib.gdn_prefill_chunked.restype = ctypes.c_int
 _lib.gdn_prefill_chunked.argtypes = _lib.gdn_prefill.argtypes
 _lib.gdn_prefill_fused.restype = ctypes.c_int
 _lib.gdn_prefill_fused.argtypes = _lib.gdn_prefill.argtypes
+_lib.gdn_prefill_stream.restype = ctypes.c_int
+_lib.gdn_prefill_stream.argtypes = _lib.gdn_prefill.argtypes
 _lib.gdn_prefill_recurrent.restype = ctypes.c_int
 _lib.gdn_prefill_recurrent.argtypes = [_P] * 10 + [_I] * 7 + [_F, _P, _P]
 _lib.gdn_prefill_static.restype = ctypes.c_int
@@ -167,12 +170,13 @@ def gdn_prefill(q, k, v, g, beta, cu_seqlens, init_state, final_state, slot_idx,
                 workspace, max_seqlen_hint=0, chunk=64, dev_status=None, route="auto"):
     """Prefill over packed sequences.  ``workspace`` is a uint8 CUDA tensor.  ``route`` picks the
     entry point: "auto" = gdn_prefill (routes by length), "chunked" = gdn_prefill_chunked (three
-    launches), "fused" = gdn_prefill_fused (one cooperative launch)."""
+    launches), "fused" = gdn_prefill_fused (one cooperative launch), "stream" = gdn_prefill_stream
+    (three launches, persistent state pass)."""
     T, Hqk, dk = q.shape
     _, Hv, dv = v.shape
     N = cu_seqlens.shape[0] - 1
     fn = {"auto": _lib.gdn_prefill, "chunked": _lib.gdn_prefill_chunked,
-          "fused": _lib.gdn_prefill_fused}[route]
+          "fused": _lib.gdn_prefill_fused, "stream": _lib.gdn_prefill_stream}[route]
     rc = fn(
         _dev(q, torch.bfloat16, "q"), _dev(k, torch.bfloat16, "k"), _dev(v, torch.bfloat16, "v"),
         _dev(g, torch.float32, "g"), _dev(beta, torch.float32, "beta"),

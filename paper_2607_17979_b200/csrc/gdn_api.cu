@@ -156,7 +156,9 @@ int gdn_prefill_recurrent(const void* q, const void* k, const void* v, const flo
 }
 
 namespace {
-int prefill_chunked_impl(bool fused, const void* q, const void* k, const void* v, const float* g,
+enum PrefillRoute { kRouteChunked, kRouteFused, kRouteStream };
+
+int prefill_chunked_impl(PrefillRoute route, const void* q, const void* k, const void* v, const float* g,
                          const float* beta, const int32_t* cu_seqlens, const float* init_state,
                          float* final_state, const int32_t* slot_idx, void* o, int32_t T, int32_t N,
                          int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv, int32_t chunk,
@@ -182,8 +184,10 @@ int prefill_chunked_impl(bool fused, const void* q, const void* k, const void* v
     p.dev_status = dev_status;
     cp.ws = static_cast<uint8_t*>(workspace);
     cp.lay = gdn::workspace_layout(T, N, Hv);
-    return cuda_status(fused ? gdn::launch_prefill_fused(cp, static_cast<cudaStream_t>(stream))
-                             : gdn::launch_prefill_chunked(cp, static_cast<cudaStream_t>(stream)));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return cuda_status(route == kRouteFused    ? gdn::launch_prefill_fused(cp, st)
+                       : route == kRouteStream ? gdn::launch_prefill_stream(cp, st)
+                                               : gdn::launch_prefill_chunked(cp, st));
 }
 }  // namespace
 
@@ -194,7 +198,7 @@ int gdn_prefill_chunked(const void* q, const void* k, const void* v, const float
                         int32_t chunk, int32_t num_slots, float scale, void* workspace,
                         size_t workspace_bytes, int32_t* dev_status, void* stream) {
     (void)max_seqlen_hint;
-    return prefill_chunked_impl(false, q, k, v, g, beta, cu_seqlens, init_state, final_state,
+    return prefill_chunked_impl(kRouteChunked, q, k, v, g, beta, cu_seqlens, init_state, final_state,
                                 slot_idx, o, T, N, Hqk, Hv, dk, dv, chunk, num_slots, scale,
                                 workspace, workspace_bytes, dev_status, stream);
 }
@@ -206,7 +210,19 @@ int gdn_prefill_fused(const void* q, const void* k, const void* v, const float* 
                       int32_t chunk, int32_t num_slots, float scale, void* workspace,
                       size_t workspace_bytes, int32_t* dev_status, void* stream) {
     (void)max_seqlen_hint;
-    return prefill_chunked_impl(true, q, k, v, g, beta, cu_seqlens, init_state, final_state,
+    return prefill_chunked_impl(kRouteFused, q, k, v, g, beta, cu_seqlens, init_state, final_state,
+                                slot_idx, o, T, N, Hqk, Hv, dk, dv, chunk, num_slots, scale,
+                                workspace, workspace_bytes, dev_status, stream);
+}
+
+int gdn_prefill_stream(const void* q, const void* k, const void* v, const float* g,
+                       const float* beta, const int32_t* cu_seqlens, const float* init_state,
+                       float* final_state, const int32_t* slot_idx, void* o, int32_t T, int32_t N,
+                       int32_t max_seqlen_hint, int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv,
+                       int32_t chunk, int32_t num_slots, float scale, void* workspace,
+                       size_t workspace_bytes, int32_t* dev_status, void* stream) {
+    (void)max_seqlen_hint;
+    return prefill_chunked_impl(kRouteStream, q, k, v, g, beta, cu_seqlens, init_state, final_state,
                                 slot_idx, o, T, N, Hqk, Hv, dk, dv, chunk, num_slots, scale,
                                 workspace, workspace_bytes, dev_status, stream);
 }
@@ -245,8 +261,13 @@ int gdn_prefill(const void* q, const void* k, const void* v, const float* g, con
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
     }
-    const bool few_units = static_cast<long long>(N) * Hv <= sms / 3 && longest > 16 * gdn::kChunk;
-    return prefill_chunked_impl(coop && few_units, q, k, v, g, beta, cu_seqlens, init_state,
+    const long long units = static_cast<long long>(N) * Hv;
+    const bool few_units = units <= sms / 3 && longest > 16 * gdn::kChunk;
+    // Many more units than SMs (many short sequences): the persistent state pass, which does not
+    // pay a CTA start, a pipeline fill and a drain per unit.
+    const bool many_units = units >= 4LL * sms;
+    const PrefillRoute route = coop && few_units ? kRouteFused : many_units ? kRouteStream : kRouteChunked;
+    return prefill_chunked_impl(route, q, k, v, g, beta, cu_seqlens, init_state,
                                 final_state, slot_idx, o, T, N, Hqk, Hv, dk, dv, chunk, num_slots,
                                 scale, workspace, workspace_bytes, dev_status, stream);
 }

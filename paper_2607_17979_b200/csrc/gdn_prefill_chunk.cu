@@ -477,13 +477,19 @@ bool make_prefill_tensor_maps(TensorMaps* maps, const PrefillParams& p) {
            make_token_map(&maps->v, p.v, p.T, static_cast<int64_t>(p.Hv) * kD);
 }
 
-cudaError_t launch_prefill_chunked(const ChunkedParams& cp, cudaStream_t stream) {
-    const PrefillParams& p = cp.p;
+cudaError_t launch_prefill_intra(const TensorMaps& maps, const ChunkedParams& cp, cudaStream_t stream) {
     cudaError_t e = cudaFuncSetAttribute(prefill_intra_kernel,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kIntraSmem);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(prefill_state_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kStateSmem);
+    dim3 grid(cp.lay.max_chunks, cp.p.Hv);
+    prefill_intra_kernel<<<grid, kIntraThreads, kIntraSmem, stream>>>(maps, cp.p, cp.ws, cp.lay);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_prefill_chunked(const ChunkedParams& cp, cudaStream_t stream) {
+    const PrefillParams& p = cp.p;
+    cudaError_t e = cudaFuncSetAttribute(prefill_state_kernel,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, kStateSmem);
     if (e != cudaSuccess) return e;
     TensorMaps maps;
     if (!make_prefill_tensor_maps(&maps, p)) return cudaErrorInvalidValue;
@@ -493,9 +499,7 @@ cudaError_t launch_prefill_chunked(const ChunkedParams& cp, cudaStream_t stream)
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (cp.lay.max_chunks > 0) {
-        dim3 grid(cp.lay.max_chunks, p.Hv);
-        prefill_intra_kernel<<<grid, kIntraThreads, kIntraSmem, stream>>>(maps, p, cp.ws, cp.lay);
-        e = cudaGetLastError();
+        e = launch_prefill_intra(maps, cp, stream);
         if (e != cudaSuccess) return e;
     }
     prefill_state_kernel<<<p.N * p.Hv, kStateThreads, kStateSmem, stream>>>(maps, p, cp.ws, cp.lay);

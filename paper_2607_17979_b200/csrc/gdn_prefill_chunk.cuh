@@ -100,5 +100,11 @@ struct ChunkedParams {
 cudaError_t launch_prefill_chunked(const ChunkedParams& cp, cudaStream_t stream);
 // One cooperative launch: some CTAs produce the records, the others run the state pass behind them.
 cudaError_t launch_prefill_fused(const ChunkedParams& cp, cudaStream_t stream);
+// Three launches with a persistent state pass: CTAs walk lists of (sequence, v-head) units and
+// stream their records without draining between units (for batches with many more units than SMs).
+cudaError_t launch_prefill_stream(const ChunkedParams& cp, cudaStream_t stream);
+// Pieces shared by the launchers: the prep kernel that also ranks the sequences by chunk count
+// (longest first) and clears the queues and flags; the intra-chunk kernel over all items.
+cudaError_t launch_prefill_ranked_prep(const ChunkedParams& cp, cudaStream_t stream);
 
 }  // namespace gdn

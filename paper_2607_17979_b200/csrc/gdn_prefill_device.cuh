@@ -33,6 +33,8 @@ struct TensorMaps {
 };
 // Host side: 2-D maps over the packed q, k, v (64 x 64 boxes, 128B swizzle); false on failure.
 bool make_prefill_tensor_maps(TensorMaps* maps, const PrefillParams& p);
+// Launch of the intra-chunk kernel over every (chunk, v-head) item of the batch.
+cudaError_t launch_prefill_intra(const TensorMaps& maps, const ChunkedParams& cp, cudaStream_t stream);
 
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;

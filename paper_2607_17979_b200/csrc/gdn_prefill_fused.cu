@@ -599,6 +599,13 @@ prefill_fused_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
 // =============================================================================================
 // host side
 // =============================================================================================
+cudaError_t launch_prefill_ranked_prep(const ChunkedParams& cp, cudaStream_t stream) {
+    prefill_fused_prep_kernel<<<1, kFPrepThreads, 0, stream>>>(cp.p.cu_seqlens, cp.p.T, cp.p.N,
+                                                               cp.p.Hv, cp.ws, cp.lay,
+                                                               cp.p.dev_status);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_prefill_fused(const ChunkedParams& cp, cudaStream_t stream) {
     const PrefillParams& p = cp.p;
     int dev = 0, sms = 0, coop = 0;
@@ -613,9 +620,7 @@ cudaError_t launch_prefill_fused(const ChunkedParams& cp, cudaStream_t stream) {
     TensorMaps maps;
     if (!make_prefill_tensor_maps(&maps, p)) return cudaErrorInvalidValue;
 
-    prefill_fused_prep_kernel<<<1, kFPrepThreads, 0, stream>>>(p.cu_seqlens, p.T, p.N, p.Hv, cp.ws,
-                                                               cp.lay, p.dev_status);
-    e = cudaGetLastError();
+    e = launch_prefill_ranked_prep(cp, stream);
     if (e != cudaSuccess) return e;
 
     // How many CTAs run the state pass: measured best near 0.43 of the SMs when there are more

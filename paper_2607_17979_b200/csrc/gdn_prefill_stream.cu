@@ -1,0 +1,450 @@
+// Inter-chunk state pass as a PERSISTENT kernel: one CTA per SM walks a fixed list of
+// (sequence, v-head) units and streams their chunk records through one two-stage pipeline that
+// does not drain between units.
+//
+// The one-CTA-per-unit state kernel pays, for every unit, a launch slot, barrier and TMEM set-up,
+// the first record's memory latency and the tail of its last chunk; with thousands of short
+// units (many short sequences) that overhead is longer than the chunk steps themselves.  Here
+//   * warp 9 (loader) copies records and K tiles in unit order, running up to two chunks ahead
+//     of the consumers and straight across unit boundaries;
+//   * warp 8 (issuer) issues every tcgen05.mma;
+//   * warps 0-7 (epilogue) carry the dependent chain  D1 = S W^T -> U = U~ - D1 ->
+//     S_acc += (U decayed)^T K -> refresh, and turn Y = S Qg^T + U P^T into o rows.
+// The three roles never meet at a CTA barrier inside the loop: each derives the same unit list
+// (unit = blockIdx.x + i * gridDim.x over the rank-sorted units, longest sequences first) and the
+// same running chunk count, from which every mbarrier parity follows.  Every barrier phase is
+// consumed by its waiter before the next one can complete (a parity wait cannot tell a barrier
+// that is two phases ahead), which is why the state hand-over after a unit's last chunk is
+// omitted rather than left unconsumed.
+//
+// The fp32 master state lives in TMEM as the accumulator of the state product, pre-scaled by the
+// next chunk's e^{b_C} (same scheme as the fused kernel's state role).
+#include "gdn_prefill_device.cuh"
+
+namespace gdn {
+
+constexpr int kSEpiWarps = 8;
+constexpr int kSEpiThreads = kSEpiWarps * 32;
+constexpr int kSIssueWarp = kSEpiWarps;
+constexpr int kSLoadWarp = kSEpiWarps + 1;
+constexpr int kStreamThreads = kSEpiThreads + 64;
+constexpr uint32_t kStreamSmem = 2 * kStageBytes + 16384 + 1024;
+
+namespace {
+
+// What every role needs to know about one unit; derived identically by each of them.
+struct UnitInfo {
+    int n, hv, hqk, c_first, nc, seq_t0, seq_len, slot;
+    bool skip;          // invalid sequence, padding / out-of-range slot, or no chunks
+    bool bad_seq, bad_slot;
+};
+
+__device__ __forceinline__ UnitInfo unit_info(const PrefillParams& p, const uint8_t* ws,
+                                              const WorkspaceLayout& lay, int unit) {
+    const int32_t* seq_first = reinterpret_cast<const int32_t*>(ws + lay.seq_first);
+    const int32_t* seq_bad = reinterpret_cast<const int32_t*>(ws + lay.seq_bad);
+    const int32_t* seq_by_rank = reinterpret_cast<const int32_t*>(ws + lay.seq_by_rank);
+    UnitInfo u;
+    const int rank = unit / p.Hv;
+    u.hv = unit - rank * p.Hv;
+    u.n = seq_by_rank[rank];
+    u.hqk = u.hv / (p.Hv / p.Hqk);
+    u.c_first = seq_first[u.n];
+    u.nc = seq_first[u.n + 1] - u.c_first;
+    u.seq_t0 = p.cu_seqlens[u.n];
+    u.seq_len = p.cu_seqlens[u.n + 1] - u.seq_t0;
+    u.slot = p.slot_idx ? p.slot_idx[u.n] : u.n;
+    u.bad_seq = seq_bad[u.n] != 0;
+    u.bad_slot = u.slot < 0 || u.slot >= p.num_slots;
+    u.skip = u.bad_seq || u.bad_slot || u.nc == 0;
+    return u;
+}
+
+}  // namespace
+
+__global__ void __launch_bounds__(kStreamThreads, 1)
+prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const PrefillParams p,
+                            uint8_t* ws, const WorkspaceLayout lay) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                               ~static_cast<uintptr_t>(1023));
+    __shared__ uint64_t bar_full[2], bar_free[2], bar_d1, bar_d4, bar_y, bar_s, bar_u;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_flag;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int half = (warp >> 2) & 1;                 // which half of the columns this thread owns
+    const int dv = (warp & 3) * 32 + lane;            // TMEM lane = state row
+    const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    const int total_units = p.N * p.Hv;
+
+    if (tid == 0) {
+        mbar_init(&bar_full[0], 1);
+        mbar_init(&bar_full[1], 1);
+        mbar_init(&bar_free[0], kSEpiWarps + 1);     // the epilogue warps + the chunk's last product
+        mbar_init(&bar_free[1], kSEpiWarps + 1);
+        mbar_init(&bar_d1, 1);
+        mbar_init(&bar_d4, 1);
+        mbar_init(&bar_y, 1);
+        mbar_init(&bar_s, kSEpiWarps);
+        mbar_init(&bar_u, kSEpiWarps);
+        abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == kSIssueWarp) {
+        tmem_alloc(&tmem_base_s, kStateTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = tmem_base_s;
+    volatile int* abortp = &abort_flag;
+
+    // gc = chunks of earlier units of this CTA; chunk j of the current unit is chunk g = gc + j of
+    // the CTA's stream: stage g & 1, phase g >> 1 of bar_full / bar_free of that stage, phase g of
+    // bar_d1 / bar_d4 / bar_y / bar_u and of bar_s (one state hand-over per chunk: the initial one
+    // and one after every chunk but the unit's last).
+    uint32_t gc = 0;
+
+    if (warp == kSLoadWarp) {
+        // ===================== loader: records and K tiles, in stream order
+        if (lane == 0) {
+            const size_t rec_stride = static_cast<size_t>(p.Hv) * kRecBytes;
+            bool live = true;
+            for (int unit = blockIdx.x; unit < total_units && live; unit += gridDim.x) {
+                const UnitInfo u = unit_info(p, ws, lay, unit);
+                if (u.skip) continue;
+                const uint8_t* records =
+                    ws + lay.records + (static_cast<size_t>(u.c_first) * p.Hv + u.hv) * kRecBytes;
+                for (int j = 0; j < u.nc; ++j) {
+                    const uint32_t g = gc + j;
+                    const int st = g & 1;
+                    // the stage held chunk g - 2: free once that chunk's last product has retired
+                    // and every epilogue warp is done with its record
+                    if (g >= 2 && !wait_or_abort(&bar_free[st], ((g - 2) >> 1) & 1u, abortp)) {
+                        live = false;
+                        break;
+                    }
+                    uint8_t* base = smem + st * kStageBytes;
+                    mbar_expect_tx(&bar_full[st], kRecBytes + 16384);
+                    bulk_load(base + kS_Rec, records + j * rec_stride, kRecBytes, &bar_full[st]);
+                    tma_load_2d(base + kS_K, &maps.k, u.hqk * kD, u.seq_t0 + j * kChunk, &bar_full[st]);
+                    tma_load_2d(base + kS_K + 8192, &maps.k, u.hqk * kD + 64, u.seq_t0 + j * kChunk,
+                                &bar_full[st]);
+                }
+                gc += u.nc;
+            }
+        }
+        __syncwarp();
+    } else if (warp == kSIssueWarp) {
+        // ===================== issuer: tensor-core instructions
+        if (lane == 0) {
+            const uint32_t id64 = make_idesc_bf16(128, 64, false, false);
+            const uint32_t id128mn = make_idesc_bf16(128, 128, false, true);
+            const uint32_t sRec0 = smem_u32(smem + kS_Rec), sRec1 = sRec0 + kStageBytes;
+            const uint64_t dW0 = make_sdesc_sw128(sRec0 + kRecW, 16, 1024);
+            const uint64_t dQ0 = make_sdesc_sw128(sRec0 + kRecQg, 16, 1024);
+            const uint64_t dP0 = make_sdesc_sw128(sRec0 + kRecP, 16, 1024);
+            const uint64_t dK0 = make_sdesc_sw128(sRec0 + kS_K, 8192, 1024);
+            const uint64_t dW1 = make_sdesc_sw128(sRec1 + kRecW, 16, 1024);
+            const uint64_t dQ1 = make_sdesc_sw128(sRec1 + kRecQg, 16, 1024);
+            const uint64_t dP1 = make_sdesc_sw128(sRec1 + kRecP, 16, 1024);
+            const uint64_t dK1 = make_sdesc_sw128(sRec1 + kS_K, 8192, 1024);
+            const uint32_t tS = tmem + kT_S, tD1 = tmem + kT_D1, tD4 = tmem + kT_D4;
+            bool live = true;
+            for (int unit = blockIdx.x; unit < total_units && live; unit += gridDim.x) {
+                const UnitInfo u = unit_info(p, ws, lay, unit);
+                if (u.skip) continue;
+                for (int j = 0; j < u.nc; ++j) {
+                    const uint32_t g = gc + j;
+                    const int st = g & 1;
+                    const uint64_t w = st ? dW1 : dW0, qg = st ? dQ1 : dQ0, pp = st ? dP1 : dP0,
+                                   kk = st ? dK1 : dK0;
+                    const uint32_t tY = tmem + kT_Y + st * 64;
+                    if (!wait_or_abort(&bar_full[st], (g >> 1) & 1u, abortp) ||
+                        !wait_or_abort(&bar_s, g & 1u, abortp)) {      // bf16 S of this chunk in TMEM
+                        live = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    // D1 = S W^T  (on the chain); k-step ks reads 16 dk: 32 bytes inside a half
+                    mma_ts_c<false>(tD1, tS, w, id64);
+                    mma_ts_c<true>(tD1, tS + 8, sdesc_advance(w, 32), id64);
+                    mma_ts_c<true>(tD1, tS + 16, sdesc_advance(w, 64), id64);
+                    mma_ts_c<true>(tD1, tS + 24, sdesc_advance(w, 96), id64);
+                    mma_ts_c<true>(tD1, tS + 32, sdesc_advance(w, 8192), id64);
+                    mma_ts_c<true>(tD1, tS + 40, sdesc_advance(w, 8192 + 32), id64);
+                    mma_ts_c<true>(tD1, tS + 48, sdesc_advance(w, 8192 + 64), id64);
+                    mma_ts_c<true>(tD1, tS + 56, sdesc_advance(w, 8192 + 96), id64);
+                    mma_commit(&bar_d1);
+                    // Y = S Qg^T  (off the chain)
+                    mma_ts_c<false>(tY, tS, qg, id64);
+                    mma_ts_c<true>(tY, tS + 8, sdesc_advance(qg, 32), id64);
+                    mma_ts_c<true>(tY, tS + 16, sdesc_advance(qg, 64), id64);
+                    mma_ts_c<true>(tY, tS + 24, sdesc_advance(qg, 96), id64);
+                    mma_ts_c<true>(tY, tS + 32, sdesc_advance(qg, 8192), id64);
+                    mma_ts_c<true>(tY, tS + 40, sdesc_advance(qg, 8192 + 32), id64);
+                    mma_ts_c<true>(tY, tS + 48, sdesc_advance(qg, 8192 + 64), id64);
+                    mma_ts_c<true>(tY, tS + 56, sdesc_advance(qg, 8192 + 96), id64);
+                    if (!wait_or_abort(&bar_u, g & 1u, abortp)) {         // U operands in TMEM
+                        live = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    // S_acc (= e^{b_C} S, prepared by the epilogue) += (U decayed, hi + lo) K
+                    // (K tile MN-major: 16 tokens = 2048 bytes)
+                    mma_ts_c<true>(tD4, tmem + kT_Us, kk, id128mn);
+                    mma_ts_c<true>(tD4, tmem + kT_Us + 8, sdesc_advance(kk, 2048), id128mn);
+                    mma_ts_c<true>(tD4, tmem + kT_Us + 16, sdesc_advance(kk, 4096), id128mn);
+                    mma_ts_c<true>(tD4, tmem + kT_Us + 24, sdesc_advance(kk, 6144), id128mn);
+                    mma_ts_c<true>(tD4, tmem + kT_UsLo, kk, id128mn);
+                    mma_ts_c<true>(tD4, tmem + kT_UsLo + 8, sdesc_advance(kk, 2048), id128mn);
+                    mma_ts_c<true>(tD4, tmem + kT_UsLo + 16, sdesc_advance(kk, 4096), id128mn);
+                    mma_ts_c<true>(tD4, tmem + kT_UsLo + 24, sdesc_advance(kk, 6144), id128mn);
+                    mma_commit(&bar_d4);
+                    // Y += U P^T
+                    mma_ts_c<true>(tY, tmem + kT_U, pp, id64);
+                    mma_ts_c<true>(tY, tmem + kT_U + 8, sdesc_advance(pp, 32), id64);
+                    mma_ts_c<true>(tY, tmem + kT_U + 16, sdesc_advance(pp, 64), id64);
+                    mma_ts_c<true>(tY, tmem + kT_U + 24, sdesc_advance(pp, 96), id64);
+                    mma_commit(&bar_y);
+                    mma_commit(&bar_free[st]);
+                }
+                gc += u.nc;
+            }
+        }
+        __syncwarp();
+    } else {
+        // ===================== epilogue warps: U, the state refresh (the dependent chain), o rows
+        auto hand_over = [&](uint64_t* bar) {     // after tcgen05.st: publish to the issuing lane
+            tmem_wait_st();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar);
+        };
+        const uint32_t tSacc = tmem + kT_D4 + lane_base + half * 64;     // this thread's 64 columns
+        const uint32_t tSbf = tmem + kT_S + lane_base + half * 32;
+        // 16 state columns at a time: fp32 values v[] -> bf16 copy, and gamma * v -> master
+        auto put_state = [&](const int c0, const float (&v)[16], const float gamma) {
+            uint32_t pk[8], sc[16];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) pk[i] = pack_bf16(v[2 * i], v[2 * i + 1]);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) sc[i] = __float_as_uint(gamma * v[i]);
+            tmem_st8(tSbf + (c0 >> 1), pk);
+            tmem_st16(tSacc + c0, sc);
+        };
+        // The o rows of a chunk are produced one chunk later, in two parts that fit the two waits
+        // of the chain: (A) scale, round, transpose into shared memory; (B) whole rows in 16-byte
+        // pieces.  `pend_*` describe the chunk whose rows are still owed (it may belong to the
+        // previous unit).
+        bool pend = false;
+        __nv_bfloat16* pend_og = nullptr;
+        int pend_len = 0;
+        uint32_t pend_y = 0;
+        const size_t tok_stride = static_cast<size_t>(p.Hv) * kD;
+        auto outputs_stage = [&]() {
+            __nv_bfloat16* sO = reinterpret_cast<__nv_bfloat16*>(smem + kS_Out);
+#pragma unroll
+            for (int c0 = 0; c0 < 32; c0 += 16) {
+                uint32_t x[16];
+                tmem_ld16(pend_y + lane_base + half * 32 + c0, x);
+                tmem_wait_ld();
+#pragma unroll
+                for (int jj = 0; jj < 16; ++jj)
+                    sO[(half * 32 + c0 + jj) * kD + dv] =
+                        __float2bfloat16(p.scale * __uint_as_float(x[jj]));
+            }
+        };
+        auto outputs_flush = [&]() {
+            const __nv_bfloat16* sO = reinterpret_cast<const __nv_bfloat16*>(smem + kS_Out);
+#pragma unroll
+            for (int it = 0; it < 4; ++it) {
+                const int row = it * 16 + (tid >> 4), piece = tid & 15;
+                if (row < pend_len)
+                    *reinterpret_cast<uint4*>(pend_og + row * tok_stride + piece * 8) =
+                        *reinterpret_cast<const uint4*>(sO + row * kD + piece * 8);
+            }
+        };
+
+        bool ok = true;
+        auto await = [&](uint64_t* bar, uint32_t parity) {   // bounded wait + tcgen05 fence
+            if (ok && !warp_wait_or_abort(bar, parity, abortp)) ok = false;
+            tc_fence_after_sync();
+        };
+        // Every warp runs every group barrier and hand-over below, also after a wait has failed
+        // (ok == false: later waits and all work are skipped), so that no warp is ever left alone
+        // at a barrier.
+        for (int unit = blockIdx.x; unit < total_units; unit += gridDim.x) {
+            const UnitInfo u = unit_info(p, ws, lay, unit);
+            const size_t tile_off = (static_cast<size_t>(u.bad_slot ? 0 : u.slot) * p.Hv + u.hv) * (kD * kD) +
+                                    static_cast<size_t>(dv) * kD + half * 64;
+            if (u.skip) {
+                if (u.bad_seq) continue;
+                if (u.bad_slot) {          // padding / out-of-range slot: zero rows, no state
+                    if (u.slot >= p.num_slots && tid == 0) report(p.dev_status, kDevBadSlot);
+                    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+                    for (int idx = tid; idx < u.seq_len * 16; idx += kSEpiThreads)
+                        *reinterpret_cast<uint4*>(p.o + (static_cast<size_t>(u.seq_t0 + (idx >> 4)) * p.Hv + u.hv) * kD +
+                                                  (idx & 15) * 8) = zero;
+                } else {                   // empty sequence: the state passes through untouched
+#pragma unroll 4
+                    for (int j = 0; j < 64; j += 4) {
+                        const float4 x = p.init_state
+                                             ? *reinterpret_cast<const float4*>(p.init_state + tile_off + j)
+                                             : make_float4(0.f, 0.f, 0.f, 0.f);
+                        *reinterpret_cast<float4*>(p.final_state + tile_off + j) = x;
+                    }
+                }
+                continue;
+            }
+            const int nc = u.nc;
+            // the unit's initial state: bf16 copy + master pre-scaled by chunk 0's e^{b_C}
+            await(&bar_full[gc & 1], (gc >> 1) & 1u);
+            if (ok) {
+                const float g0 = reinterpret_cast<const float*>(smem + (gc & 1) * kStageBytes + kS_Rec +
+                                                                kRecGammaC)[0];
+#pragma unroll 1
+                for (int c0 = 0; c0 < 64; c0 += 16) {
+                    float v[16];
+#pragma unroll
+                    for (int i = 0; i < 16; i += 4) {
+                        const float4 x = p.init_state
+                                             ? *reinterpret_cast<const float4*>(p.init_state + tile_off + c0 + i)
+                                             : make_float4(0.f, 0.f, 0.f, 0.f);
+                        v[i] = x.x; v[i + 1] = x.y; v[i + 2] = x.z; v[i + 3] = x.w;
+                    }
+                    put_state(c0, v, g0);
+                }
+            }
+            hand_over(&bar_s);
+            for (int j = 0; j < nc; ++j) {
+                const uint32_t g = gc + j;
+                const int st = g & 1;
+                const uint8_t* base = smem + st * kStageBytes;
+                if (pend) {     // part A of the previous chunk's rows, while D1 is in flight
+                    await(&bar_y, (g - 1) & 1u);
+                    epi_group_sync();
+                    if (ok) outputs_stage();
+                }
+                await(&bar_full[st], (g >> 1) & 1u);
+                await(&bar_d1, g & 1u);
+                if (ok) {   // U^T[dv][c] = U~^T - D1 for the thread's 32 tokens [32*half, 32*half+32)
+                    const float4* sU = reinterpret_cast<const float4*>(base + kS_Rec + kRecU);
+                    const float* sdec = reinterpret_cast<const float*>(base + kS_Rec + kRecDecay);
+#pragma unroll
+                    for (int c0 = 0; c0 < 32; c0 += 16) {
+                        const int cb = half * 32 + c0;
+                        uint32_t x[16];
+                        tmem_ld16(tmem + kT_D1 + lane_base + cb, x);
+                        tmem_wait_ld();
+                        uint32_t pu[8], ph[8], pl[8];
+#pragma unroll
+                        for (int q4 = 0; q4 < 4; ++q4) {
+                            const float4 ut = sU[((cb >> 2) + q4) * kD + dv];
+                            const float4 dd = *reinterpret_cast<const float4*>(sdec + cb + 4 * q4);
+                            const float u0 = ut.x - __uint_as_float(x[4 * q4 + 0]);
+                            const float u1 = ut.y - __uint_as_float(x[4 * q4 + 1]);
+                            const float u2 = ut.z - __uint_as_float(x[4 * q4 + 2]);
+                            const float u3 = ut.w - __uint_as_float(x[4 * q4 + 3]);
+                            const float s0 = u0 * dd.x, s1 = u1 * dd.y, s2 = u2 * dd.z, s3 = u3 * dd.w;
+                            pu[2 * q4] = pack_bf16(u0, u1);
+                            pu[2 * q4 + 1] = pack_bf16(u2, u3);
+                            ph[2 * q4] = pack_bf16(s0, s1);
+                            ph[2 * q4 + 1] = pack_bf16(s2, s3);
+                            pl[2 * q4] = pack_bf16(s0 - __uint_as_float(ph[2 * q4] << 16),
+                                                   s1 - __uint_as_float(ph[2 * q4] & 0xffff0000u));
+                            pl[2 * q4 + 1] = pack_bf16(s2 - __uint_as_float(ph[2 * q4 + 1] << 16),
+                                                       s3 - __uint_as_float(ph[2 * q4 + 1] & 0xffff0000u));
+                        }
+                        tmem_st8(tmem + kT_Us + lane_base + (cb >> 1), ph);
+                        tmem_st8(tmem + kT_UsLo + lane_base + (cb >> 1), pl);
+                        tmem_st8(tmem + kT_U + lane_base + (cb >> 1), pu);
+                    }
+                }
+                hand_over(&bar_u);
+                if (pend) {     // part B, while this chunk's state product is in flight
+                    epi_group_sync();
+                    if (ok) outputs_flush();
+                }
+                pend = true;
+                pend_og = p.o + (static_cast<size_t>(u.seq_t0 + j * kChunk) * p.Hv + u.hv) * kD;
+                pend_len = min(kChunk, u.seq_len - j * kChunk);
+                pend_y = tmem + kT_Y + st * 64;
+                const bool last = j + 1 == nc;
+                if (!last) await(&bar_full[st ^ 1], ((g + 1) >> 1) & 1u);   // next record's e^{b_C}
+                await(&bar_d4, g & 1u);
+                if (ok) {   // the master now holds S(j+1): refresh the bf16 copy, pre-scale the master
+                    const float gn = last ? 1.f
+                                          : reinterpret_cast<const float*>(smem + (st ^ 1) * kStageBytes +
+                                                                           kS_Rec + kRecGammaC)[0];
+#pragma unroll 2
+                    for (int c0 = 0; c0 < 64; c0 += 16) {
+                        uint32_t x[16];
+                        tmem_ld16(tSacc + c0, x);
+                        tmem_wait_ld();
+                        float v[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(x[i]);
+                        if (!last) {
+                            put_state(c0, v, gn);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 16; i += 4)
+                                *reinterpret_cast<float4*>(p.final_state + tile_off + c0 + i) =
+                                    make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                        }
+                    }
+                }
+                if (lane == 0) mbar_arrive(&bar_free[st]);     // this warp is done with the stage
+                if (!last) hand_over(&bar_s);
+            }
+            gc += nc;
+        }
+        if (pend) {     // the rows of the stream's last chunk
+            await(&bar_y, (gc - 1) & 1u);
+            epi_group_sync();
+            if (ok) outputs_stage();
+            epi_group_sync();
+            if (ok) outputs_flush();
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (abort_flag != 0 && warp == kSIssueWarp && lane == 0) {
+        report(p.dev_status, kDevTimeout);
+        // let copies already in flight land before the CTA's shared memory goes away
+        mbar_wait(&bar_full[0], 0, 1u << 12);
+        mbar_wait(&bar_full[1], 0, 1u << 12);
+    }
+    __syncwarp();
+    if (warp == kSIssueWarp) tmem_dealloc(tmem, kStateTmemCols);
+}
+
+// Prep (chunk table + sequences ranked by chunk count) is the fused path's; then the intra-chunk
+// kernel over all items; then this kernel on min(units, SMs) CTAs.
+cudaError_t launch_prefill_stream(const ChunkedParams& cp, cudaStream_t stream) {
+    const PrefillParams& p = cp.p;
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    e = cudaFuncSetAttribute(prefill_state_stream_kernel,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmem);
+    if (e != cudaSuccess) return e;
+    TensorMaps maps;
+    if (!make_prefill_tensor_maps(&maps, p)) return cudaErrorInvalidValue;
+    e = launch_prefill_ranked_prep(cp, stream);
+    if (e != cudaSuccess) return e;
+    if (cp.lay.max_chunks > 0) {
+        e = launch_prefill_intra(maps, cp, stream);
+        if (e != cudaSuccess) return e;
+    }
+    const long long units = static_cast<long long>(p.N) * p.Hv;
+    const int grid = static_cast<int>(units < sms ? units : sms);
+    prefill_state_stream_kernel<<<grid, kStreamThreads, kStreamSmem, stream>>>(maps, p, cp.ws, cp.lay);
+    return cudaGetLastError();
+}
+
+}  // namespace gdn
