@@ -111,8 +111,11 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
         if (lane == 0) {
             const size_t rec_stride = static_cast<size_t>(p.Hv) * kRecBytes;
             bool live = true;
+            // the next unit's table entries are fetched while the current unit is processed
+            UnitInfo nxt = unit_info(p, ws, lay, min(static_cast<int>(blockIdx.x), total_units - 1));
             for (int unit = blockIdx.x; unit < total_units && live; unit += gridDim.x) {
-                const UnitInfo u = unit_info(p, ws, lay, unit);
+                const UnitInfo u = nxt;
+                nxt = unit_info(p, ws, lay, min(unit + static_cast<int>(gridDim.x), total_units - 1));
                 if (u.skip) continue;
                 const uint8_t* records =
                     ws + lay.records + (static_cast<size_t>(u.c_first) * p.Hv + u.hv) * kRecBytes;
@@ -152,8 +155,11 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
             const uint64_t dK1 = make_sdesc_sw128(sRec1 + kS_K, 8192, 1024);
             const uint32_t tS = tmem + kT_S, tD1 = tmem + kT_D1, tD4 = tmem + kT_D4;
             bool live = true;
+            // the next unit's table entries are fetched while the current unit is processed
+            UnitInfo nxt = unit_info(p, ws, lay, min(static_cast<int>(blockIdx.x), total_units - 1));
             for (int unit = blockIdx.x; unit < total_units && live; unit += gridDim.x) {
-                const UnitInfo u = unit_info(p, ws, lay, unit);
+                const UnitInfo u = nxt;
+                nxt = unit_info(p, ws, lay, min(unit + static_cast<int>(gridDim.x), total_units - 1));
                 if (u.skip) continue;
                 for (int j = 0; j < u.nc; ++j) {
                     const uint32_t g = gc + j;
@@ -275,8 +281,10 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
         // Every warp runs every group barrier and hand-over below, also after a wait has failed
         // (ok == false: later waits and all work are skipped), so that no warp is ever left alone
         // at a barrier.
+        UnitInfo nxt = unit_info(p, ws, lay, min(static_cast<int>(blockIdx.x), total_units - 1));
         for (int unit = blockIdx.x; unit < total_units; unit += gridDim.x) {
-            const UnitInfo u = unit_info(p, ws, lay, unit);
+            const UnitInfo u = nxt;
+            nxt = unit_info(p, ws, lay, min(unit + static_cast<int>(gridDim.x), total_units - 1));
             const size_t tile_off = (static_cast<size_t>(u.bad_slot ? 0 : u.slot) * p.Hv + u.hv) * (kD * kD) +
                                     static_cast<size_t>(dv) * kD + half * 64;
             if (u.skip) {
