@@ -3,6 +3,7 @@ tokens to 8192 tokens in up to 57 sequences): the shape distribution of the pape
 GDN tables, on seeded synthetic inputs.  Prints one JSON object per shape and a summary line.
 
     python -m paper_2607_17979_b200.sweep [--reps 200]
+    python -m paper_2607_17979_b200.sweep --lens 144x56,128 --route stream   # one prefill shape
 
 Each shape's call is captured `GRAPH_CALLS` times into one CUDA graph, and the graph is replayed
 and timed with CUDA events: the number is device time per call including kernel launch gaps but
@@ -60,11 +61,35 @@ def _time(fn, reps):
     return e0.elapsed_time(e1) / (replays * GRAPH_CALLS) * 1e3          # microseconds
 
 
+def _prefill_row(lens, route, reps):
+    p = I.prefill_inputs(lens, 16, 32, 128, seed=I.BASE_SEED + sum(lens), init="zero")
+    t = {n: _bf16(p[n]) for n in "qkv"}
+    g, beta, cu = _dev(p["g"]), _dev(p["beta"]), _dev(p["cu_seqlens"])
+    final = torch.empty((p["N"], 32, 128, 128), dtype=torch.float32, device="cuda")
+    o = torch.empty((p["T"], 32, 128), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(api.gdn_prefill_workspace_bytes(p["T"], p["N"], 16, 32), dtype=torch.uint8,
+                     device="cuda")
+    us = _time(lambda: api.gdn_prefill(t["q"], t["k"], t["v"], g, beta, cu, None, final, None, o,
+                                       p["scale"], ws, max_seqlen_hint=max(lens), route=route), reps)
+    return {"op": "prefill", "route": route, "tokens": p["T"], "seqs": p["N"], "longest": max(lens),
+            "us": us, "tokens_per_s": p["T"] / us * 1e6}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--reps", type=int, default=200)
+    ap.add_argument("--lens", default="", help="time one prefill shape only: comma-separated "
+                    "sequence lengths, LENxCOUNT for repeats (e.g. 144x56,128)")
+    ap.add_argument("--route", default="auto", choices=["auto", "chunked", "fused", "stream"])
     args = ap.parse_args()
     rows = []
+    if args.lens:
+        lens = []
+        for part in args.lens.split(","):
+            n, _, c = part.partition("x")
+            lens += [int(n)] * (int(c) if c else 1)
+        print(json.dumps(_prefill_row(lens, args.route, max(10, args.reps // 4))))
+        return
     for B in DECODE_BATCHES:
         d = I.decode_inputs(B, 16, 32, 128, B, seed=I.BASE_SEED + B)
         t = {n: _bf16(d[n]) for n in "qkv"}
@@ -86,18 +111,7 @@ def main():
             rows.append({"op": "decode_multi", "B": B, "L": L, "layout": name, "us": us,
                          "tokens_per_s": B * L / us * 1e6})
     for lens in PREFILL_SHAPES:
-        p = I.prefill_inputs(lens, 16, 32, 128, seed=I.BASE_SEED + sum(lens), init="zero")
-        t = {n: _bf16(p[n]) for n in "qkv"}
-        g, beta, cu = _dev(p["g"]), _dev(p["beta"]), _dev(p["cu_seqlens"])
-        final = torch.empty((p["N"], 32, 128, 128), dtype=torch.float32, device="cuda")
-        o = torch.empty((p["T"], 32, 128), dtype=torch.bfloat16, device="cuda")
-        ws = torch.empty(api.gdn_prefill_workspace_bytes(p["T"], p["N"], 16, 32), dtype=torch.uint8,
-                         device="cuda")
-        us = _time(lambda: api.gdn_prefill(t["q"], t["k"], t["v"], g, beta, cu, None, final, None, o,
-                                           p["scale"], ws, max_seqlen_hint=max(lens)),
-                   max(10, args.reps // 4))
-        rows.append({"op": "prefill", "tokens": p["T"], "seqs": p["N"], "longest": max(lens),
-                     "us": us, "tokens_per_s": p["T"] / us * 1e6})
+        rows.append(_prefill_row(lens, "auto", max(10, args.reps // 4)))
     for r in rows:
         print(json.dumps(r))
     dec = [r["us"] for r in rows if r["op"] == "decode"]
