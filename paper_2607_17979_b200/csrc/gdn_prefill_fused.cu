@@ -89,20 +89,52 @@ prefill_fused_prep_kernel(const int32_t* __restrict__ cu, int32_t T, int32_t N, 
         seq_first[N] = running;
         hdr[kHdrTotalChunks] = running;
         hdr[kHdrTotalItems] = running * Hv;
-        // cnt[v] = number of sequences with more than v chunks (suffix sum of the histogram);
-        // pos[j] = number of chunks at positions < j
-        int32_t above = 0;
-        for (int v = lay.max_nc; v >= 0; --v) {
-            cnt[v] = above;
-            above += hist[v];
-        }
-        int32_t before = 0;
-        for (int j = 0; j <= lay.max_nc; ++j) {
-            pos[j] = before;
-            before += cnt[j];
-        }
+        running = 0;
     }
     __syncthreads();
+    // cnt[v] = number of sequences with more than v chunks: exclusive suffix sum of the histogram,
+    // as a block scan over tiles of the reversed index u = max_nc - v
+    for (int base = 0; base <= lay.max_nc; base += kFPrepThreads) {
+        const int u = base + tid;
+        const int32_t x = u <= lay.max_nc ? hist[lay.max_nc - u] : 0;
+        int32_t incl = x;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int32_t y = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += y;
+        }
+        if (lane == 31) warp_sums[warp] = incl;
+        __syncthreads();
+        int32_t warp_off = 0;
+        for (int w = 0; w < warp; ++w) warp_off += warp_sums[w];
+        const int32_t excl = running + warp_off + incl - x;
+        if (u <= lay.max_nc) cnt[lay.max_nc - u] = excl;
+        __syncthreads();
+        if (tid == kFPrepThreads - 1) running = excl + x;
+        __syncthreads();
+    }
+    if (tid == 0) running = 0;
+    __syncthreads();
+    // pos[j] = number of chunks at positions < j: exclusive prefix sum of cnt
+    for (int base = 0; base <= lay.max_nc; base += kFPrepThreads) {
+        const int j = base + tid;
+        const int32_t x = j <= lay.max_nc ? cnt[j] : 0;
+        int32_t incl = x;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int32_t y = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += y;
+        }
+        if (lane == 31) warp_sums[warp] = incl;
+        __syncthreads();
+        int32_t warp_off = 0;
+        for (int w = 0; w < warp; ++w) warp_off += warp_sums[w];
+        const int32_t excl = running + warp_off + incl - x;
+        if (j <= lay.max_nc) pos[j] = excl;
+        __syncthreads();
+        if (tid == kFPrepThreads - 1) running = excl + x;
+        __syncthreads();
+    }
     // rank of a sequence = its place in the order "more chunks first"; chunk j of the sequence of
     // rank r is processed at place pos[j] + r (the sequences that have a chunk j are ranks < cnt[j])
     for (int n = tid; n < N; n += kFPrepThreads) {
