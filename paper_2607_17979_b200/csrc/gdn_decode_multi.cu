@@ -111,7 +111,7 @@ __device__ __forceinline__ void zero_outputs(const DecodeMultiParams& mp, int i,
 // ---- layout 0: tile [dv][dk] -------------------------------------------------------------------
 // kPasses = 4: one CTA per tile; kPasses = 1: a tile split over four CTAs of 32 dv rows each.
 template <int kPasses>
-__global__ void __launch_bounds__(kMultiThreads, 2)
+__global__ void __launch_bounds__(kMultiThreads, kPasses == 4 ? 2 : 3)
 decode_multi_vk_kernel(const DecodeMultiParams mp) {
     __shared__ __align__(16) TokenStage st;
     const DecodeParams& p = mp.d;
@@ -188,9 +188,9 @@ decode_multi_vk_kernel(const DecodeMultiParams mp) {
 // ---- layout 1: tile [dk][dv] -------------------------------------------------------------------
 // kSplit = 1: one CTA per tile, a warp load covers one whole 512-byte row, a warp owns 16 rows.
 // kSplit = 4: four CTAs per tile, each owning 32 dv columns (columns evolve independently); a warp
-// load covers the 128-byte column share of four rows.
+// load covers the 128-byte column share of four rows.  kSplit = 2: two CTAs of 64 columns.
 template <int kSplit>
-__global__ void __launch_bounds__(kMultiThreads, 2)
+__global__ void __launch_bounds__(kMultiThreads, kSplit == 2 ? 3 : 2)
 decode_multi_kv_kernel(const DecodeMultiParams mp) {
     __shared__ __align__(16) TokenStage st;
     constexpr int kCols = kD / kSplit;            // dv columns of this CTA
@@ -302,9 +302,13 @@ cudaError_t launch_decode_multi(const DecodeMultiParams& mp, cudaStream_t stream
     const unsigned grid = static_cast<unsigned>(split ? units * 4 : units);
     if (mp.layout == 0) {
         if (split) decode_multi_vk_kernel<1><<<grid, kMultiThreads, 0, stream>>>(mp);
+        // up to four tokens half tiles at three CTAs per SM overlap loads and arithmetic better;
+        // beyond that the four independent row groups of a whole tile hide the per-token chain
+        else if (mp.L <= 4) decode_multi_vk_kernel<2><<<grid * 2, kMultiThreads, 0, stream>>>(mp);
         else decode_multi_vk_kernel<4><<<grid, kMultiThreads, 0, stream>>>(mp);
     } else {
         if (split) decode_multi_kv_kernel<4><<<grid, kMultiThreads, 0, stream>>>(mp);
+        else if (mp.L <= 2) decode_multi_kv_kernel<2><<<grid * 2, kMultiThreads, 0, stream>>>(mp);
         else decode_multi_kv_kernel<1><<<grid, kMultiThreads, 0, stream>>>(mp);
     }
     return cudaGetLastError();

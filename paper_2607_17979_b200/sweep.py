@@ -4,6 +4,7 @@ GDN tables, on seeded synthetic inputs.  Prints one JSON object per shape and a 
 
     python -m paper_2607_17979_b200.sweep [--reps 200]
     python -m paper_2607_17979_b200.sweep --lens 144x56,128 --route stream   # one prefill shape
+    python -m paper_2607_17979_b200.sweep --decode-multi 64x4                # one multi-token shape
 
 Each shape's call is captured `GRAPH_CALLS` times into one CUDA graph, and the graph is replayed
 and timed with CUDA events: the number is device time per call including kernel launch gaps but
@@ -61,6 +62,20 @@ def _time(fn, reps):
     return e0.elapsed_time(e1) / (replays * GRAPH_CALLS) * 1e3          # microseconds
 
 
+def _multi_rows(B, L, reps):
+    d = I.decode_multi_inputs(B, L, 16, 32, 128, B, seed=I.BASE_SEED + 7 * B + L)
+    t = {n: _bf16(d[n]) for n in "qkv"}
+    g, beta, pool = _dev(d["g"]), _dev(d["beta"]), _dev(d["state"])
+    o = torch.empty((B, L, 32, 128), dtype=torch.bfloat16, device="cuda")
+    out = []
+    for layout, name in ((api.STATE_VK, "vk"), (api.STATE_KV, "kv")):
+        us = _time(lambda: api.gdn_decode_multi(t["q"], t["k"], t["v"], g, beta, pool, None, o,
+                                                d["scale"], layout), reps)
+        out.append({"op": "decode_multi", "B": B, "L": L, "layout": name, "us": us,
+                    "tokens_per_s": B * L / us * 1e6})
+    return out
+
+
 def _prefill_row(lens, route, reps):
     p = I.prefill_inputs(lens, 16, 32, 128, seed=I.BASE_SEED + sum(lens), init="zero")
     t = {n: _bf16(p[n]) for n in "qkv"}
@@ -81,8 +96,15 @@ def main():
     ap.add_argument("--lens", default="", help="time one prefill shape only: comma-separated "
                     "sequence lengths, LENxCOUNT for repeats (e.g. 144x56,128)")
     ap.add_argument("--route", default="auto", choices=["auto", "chunked", "fused", "stream"])
+    ap.add_argument("--decode-multi", default="", help="time one multi-token decode shape only: "
+                    "BxL (both state orientations)")
     args = ap.parse_args()
     rows = []
+    if args.decode_multi:
+        B, _, L = args.decode_multi.partition("x")
+        for r in _multi_rows(int(B), int(L), args.reps):
+            print(json.dumps(r))
+        return
     if args.lens:
         lens = []
         for part in args.lens.split(","):
@@ -101,15 +123,7 @@ def main():
                      "state_GBps": 2 * B * 32 * 65536 / us / 1e3})
     # multi-token decode (L new tokens per sequence in one call), both state orientations
     for B, L in MULTI_SHAPES:
-        d = I.decode_multi_inputs(B, L, 16, 32, 128, B, seed=I.BASE_SEED + 7 * B + L)
-        t = {n: _bf16(d[n]) for n in "qkv"}
-        g, beta, pool = _dev(d["g"]), _dev(d["beta"]), _dev(d["state"])
-        o = torch.empty((B, L, 32, 128), dtype=torch.bfloat16, device="cuda")
-        for layout, name in ((api.STATE_VK, "vk"), (api.STATE_KV, "kv")):
-            us = _time(lambda: api.gdn_decode_multi(t["q"], t["k"], t["v"], g, beta, pool, None, o,
-                                                    d["scale"], layout), args.reps)
-            rows.append({"op": "decode_multi", "B": B, "L": L, "layout": name, "us": us,
-                         "tokens_per_s": B * L / us * 1e6})
+        rows += _multi_rows(B, L, args.reps)
     for lens in PREFILL_SHAPES:
         rows.append(_prefill_row(lens, "auto", max(10, args.reps // 4)))
     for r in rows:
