@@ -71,7 +71,7 @@ prefill_prep_kernel(const int32_t* __restrict__ cu, int32_t T, int32_t N, uint8_
 // =============================================================================================
 // K1: intra-chunk quantities, one CTA (256 threads) per (chunk, v-head); see intra_item().
 // =============================================================================================
-__global__ void __launch_bounds__(kIntraThreads, 3)
+__global__ void __launch_bounds__(kIntraThreads, 4)
 prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParams p, uint8_t* ws,
                      const WorkspaceLayout lay) {
     const int c = blockIdx.x;

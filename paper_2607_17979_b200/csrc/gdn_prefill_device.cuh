@@ -12,21 +12,23 @@ constexpr int kIntraThreads = 256;
 constexpr uint32_t kIntraTmemCols = 128;
 constexpr int kLdA = 68;               // row stride (floats) of the fp32 A / T matrix
 // Shared memory map (bytes from a 1024-aligned base).  Regions are reused as their contents die
-// so that three CTAs fit on an SM:
-//   R1  Q/K tiles.  Q halves -> Qg image (stored early) -> T_w and T_u(hi);  K halves -> W image.
-//   R2  A, then T, in fp32 plus the solve scratch -> V tile (loaded after the solve).
-//   R3  P image (stored early) -> T_u(lo).
+// so that four CTAs fit on an SM:
+//   R1  Q/K tiles.  Q half 0 -> Qg image (stored early) -> solve scratch -> T_w -> T_u(lo);
+//       Q half 1 -> Qg image -> T_u(hi);  K halves -> W image.
+//   R2  A, then T, in fp32 -> V tile (loaded after the solve).
+// The P image goes straight from registers to the record; T_u(lo) waits in registers until the
+// product that reads T_w has retired.
 constexpr uint32_t kI_QK = 0;          // 2 halves x [128 rows x 128 B]: rows 0-63 Q, 64-127 K
 constexpr uint32_t kI_Tw = 0;          // over Q half 0: T diag(beta e^b) [64 r x 64 i] bf16, K-major
-constexpr uint32_t kI_Tu = 16384;      // over Q half 1: T diag(beta) rounded to bf16 ...
+constexpr uint32_t kI_TuLo = 0;        // ... and later the bf16 remainder of T diag(beta)
+constexpr uint32_t kI_Scr = 0;         // ... and, between the two, the solve scratch, fp32 [32][40]
+constexpr uint32_t kI_Tu = 16384;      // over Q half 1: T diag(beta) rounded to bf16
 constexpr uint32_t kI_A = 32768;       // A, then T in place: fp32 [64][kLdA]
-constexpr uint32_t kI_Scr = kI_A + 64 * kLdA * 4;      // solve scratch, fp32 [32][40]
 constexpr uint32_t kI_V = 32768;       // over A: 2 halves x [64 x 128 B]
-constexpr uint32_t kI_P = 32768 + 22528;               // P image staging
-constexpr uint32_t kI_TuLo = kI_P;     // ... and the bf16 remainder of T diag(beta)
-constexpr uint32_t kI_End = kI_P + 8192;
+constexpr uint32_t kI_End = kI_A + 64 * kLdA * 4;      // 50176
 constexpr uint32_t kIntraSmem = kI_End + 1024;         // + alignment slack
-static_assert(kI_Scr + 32 * 40 * 4 <= kI_P, "solve scratch overlaps the P image");
+static_assert(32 * 40 * 4 <= 8192, "solve scratch must fit in the Q half it borrows");
+static_assert(kI_End % 1024 == 0 && 64 * kLdA * 4 >= 16384, "V tile must fit over A");
 
 struct TensorMaps {
     CUtensorMap q, k, v;
@@ -106,6 +108,8 @@ __device__ __forceinline__ void solve_unit_lower_64(float* sA, float* scr, int t
 #pragma unroll
         for (int r = 0; r < 16; ++r) blk[r * kLdA + j] = t[r];
     }
+    // the scratch borrows shared memory whose previous contents thread 0 is still bulk-storing
+    if (tid == 0) bulk_wait_read_all();
     sync();
     // ---- off-diagonal blocks on the tensor cores (mma.sync m16n8k8, 3xTF32: fp32-level accuracy)
     const int warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
@@ -308,7 +312,7 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
                     w.y = pack_bf16(val[8 * h + 2], val[8 * h + 3]);
                     w.z = pack_bf16(val[8 * h + 4], val[8 * h + 5]);
                     w.w = pack_bf16(val[8 * h + 6], val[8 * h + 7]);
-                    *reinterpret_cast<uint4*>(smem + kI_P + sw128_offset(r, (cbase >> 3) + h)) = w;
+                    *reinterpret_cast<uint4*>(rec + kRecP + sw128_offset(r, (cbase >> 3) + h)) = w;
                 }
             } else {
 #pragma unroll
@@ -336,18 +340,15 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
     tc_fence_before_sync();
     sync();
     if (tid == 0) {
-        // Qg and P are final: store them now; their shared memory is reused after the solve
+        // Qg is final: store it now; its shared memory is reused from the solve on
         bulk_store(rec + kRecQg, smem + kI_QK, 8192);
         bulk_store(rec + kRecQg + 8192, smem + kI_QK + 16384, 8192);
-        bulk_store(rec + kRecP, smem + kI_P, 8192);
         bulk_commit();
     }
 
     solve_unit_lower_64(sA, reinterpret_cast<float*>(smem + kI_Scr), tid, sync);
 
-    if (tid == 0) bulk_wait_read_all();      // the Q halves and the P image have been read out
-    sync();
-
+    uint32_t tu_lo[2][4];    // T diag(beta) - bf16(T diag(beta)), parked until T_w is dead
     {   // T (fp32, row-major) -> bf16 B operands T diag(beta e^b), T diag(beta) (hi, lo)
 #pragma unroll
         for (int it = 0; it < 2; ++it) {
@@ -362,19 +363,18 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
             const float tv[8] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
             const float gv[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
             const float ev[8] = {e0.x, e0.y, e0.z, e0.w, e1.x, e1.y, e1.z, e1.w};
-            uint32_t w[4], hi[4], lo[4];
+            uint32_t w[4], hi[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 w[j] = pack_bf16(tv[2 * j] * gv[2 * j], tv[2 * j + 1] * gv[2 * j + 1]);
                 const float u0 = tv[2 * j] * ev[2 * j], u1 = tv[2 * j + 1] * ev[2 * j + 1];
                 hi[j] = pack_bf16(u0, u1);
-                lo[j] = pack_bf16(u0 - __uint_as_float(hi[j] << 16),
-                                  u1 - __uint_as_float(hi[j] & 0xffff0000u));
+                tu_lo[it][j] = pack_bf16(u0 - __uint_as_float(hi[j] << 16),
+                                         u1 - __uint_as_float(hi[j] & 0xffff0000u));
             }
             const uint32_t off = sw128_offset(r, c8);
             *reinterpret_cast<uint4*>(smem + kI_Tw + off) = make_uint4(w[0], w[1], w[2], w[3]);
             *reinterpret_cast<uint4*>(smem + kI_Tu + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-            *reinterpret_cast<uint4*>(smem + kI_TuLo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
         }
     }
     fence_proxy_async_smem();
@@ -416,6 +416,13 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
                 *reinterpret_cast<__nv_bfloat16*>(sW + sw128_offset(cbase + j, wchunk) + wcol) =
                     __float2bfloat16(__uint_as_float(x[j]));
         }
+    }
+    // the product that read T_w has retired: its place takes the remainder of T diag(beta)
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {
+        const int idx = tid + it * kIntraThreads;
+        *reinterpret_cast<uint4*>(smem + kI_TuLo + sw128_offset(idx >> 3, idx & 7)) =
+            make_uint4(tu_lo[it][0], tu_lo[it][1], tu_lo[it][2], tu_lo[it][3]);
     }
     fence_proxy_async_smem();
     tc_fence_before_sync();
