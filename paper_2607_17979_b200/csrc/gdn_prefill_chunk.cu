@@ -203,13 +203,14 @@ prefill_state_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
                 };
                 const uint32_t id64 = make_idesc_bf16(128, 64, false, false);
                 const uint32_t id128mn = make_idesc_bf16(128, 128, false, true);
+                const uint32_t id64mn = make_idesc_bf16(128, 64, false, true);
                 // base descriptors of both stages, built once; the loop only adds offsets
                 const uint32_t sRec0 = smem_u32(smem + kS_Rec), sRec1 = sRec0 + kStageBytes;
-                const uint64_t dW0 = make_sdesc_sw128(sRec0 + kRecW, 16, 1024);
+                const uint64_t dW0 = make_sdesc_sw128(sRec0 + kRecW, 8192, 1024);
                 const uint64_t dQ0 = make_sdesc_sw128(sRec0 + kRecQg, 16, 1024);
                 const uint64_t dP0 = make_sdesc_sw128(sRec0 + kRecP, 16, 1024);
                 const uint64_t dK0 = make_sdesc_sw128(sRec0 + kS_K, 8192, 1024);
-                const uint64_t dW1 = make_sdesc_sw128(sRec1 + kRecW, 16, 1024);
+                const uint64_t dW1 = make_sdesc_sw128(sRec1 + kRecW, 8192, 1024);
                 const uint64_t dQ1 = make_sdesc_sw128(sRec1 + kRecQg, 16, 1024);
                 const uint64_t dP1 = make_sdesc_sw128(sRec1 + kRecP, 16, 1024);
                 const uint64_t dK1 = make_sdesc_sw128(sRec1 + kS_K, 8192, 1024);
@@ -224,15 +225,15 @@ prefill_state_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
                     if (!wait_or_abort(&bar_full[st], (j >> 1) & 1, abortp)) break;
                     if (!wait_or_abort(&bar_s, j & 1, abortp)) break;       // bf16 S of chunk j in TMEM
                     tc_fence_after_sync();
-                    // D1 = S W^T  (on the chain); k-step ks reads 16 dk: 32 bytes inside a half
-                    mma_ts_c<false>(tD1, tS, w, id64);
-                    mma_ts_c<true>(tD1, tS + 8, sdesc_advance(w, 32), id64);
-                    mma_ts_c<true>(tD1, tS + 16, sdesc_advance(w, 64), id64);
-                    mma_ts_c<true>(tD1, tS + 24, sdesc_advance(w, 96), id64);
-                    mma_ts_c<true>(tD1, tS + 32, sdesc_advance(w, 8192), id64);
-                    mma_ts_c<true>(tD1, tS + 40, sdesc_advance(w, 8192 + 32), id64);
-                    mma_ts_c<true>(tD1, tS + 48, sdesc_advance(w, 8192 + 64), id64);
-                    mma_ts_c<true>(tD1, tS + 56, sdesc_advance(w, 8192 + 96), id64);
+                    // D1 = S W^T  (on the chain); W is MN-major: k-step ks reads 16 dk rows = 2048 bytes
+                    mma_ts_c<false>(tD1, tS, w, id64mn);
+                    mma_ts_c<true>(tD1, tS + 8, sdesc_advance(w, 2048), id64mn);
+                    mma_ts_c<true>(tD1, tS + 16, sdesc_advance(w, 4096), id64mn);
+                    mma_ts_c<true>(tD1, tS + 24, sdesc_advance(w, 6144), id64mn);
+                    mma_ts_c<true>(tD1, tS + 32, sdesc_advance(w, 8192), id64mn);
+                    mma_ts_c<true>(tD1, tS + 40, sdesc_advance(w, 10240), id64mn);
+                    mma_ts_c<true>(tD1, tS + 48, sdesc_advance(w, 12288), id64mn);
+                    mma_ts_c<true>(tD1, tS + 56, sdesc_advance(w, 14336), id64mn);
                     mma_commit(&bar_d1);
                     if (j > 0 && j + 1 < nc) {
                         // the other stage is free once chunk j-1's last product has retired (the

@@ -23,8 +23,9 @@ namespace gdn {
 
 // One record per (chunk, v-head), written by the intra-chunk kernel in exactly the
 // byte image the state-pass kernel wants in shared memory (one linear bulk copy):
-//   [0, 16384)      W   as two K-major 128B-swizzled halves [64 tokens][64 dk] bf16
-//   [16384, 32768)  Qg  = diag(e^b) Q, same layout as W (the output's first term S0 Qg^T)
+//   [0, 16384)      W   as one MN-major 128B-swizzled tile [128 dk][64 tokens] bf16 (a row per dk)
+//   [16384, 32768)  Qg  = diag(e^b) Q as two K-major 128B-swizzled halves [64 tokens][64 dk] bf16
+//                   (the output's first term S0 Qg^T)
 //   [32768, 40960)  P   as one K-major 128B-swizzled tile   [64 r][64 i]      bf16
 //   [40960, 73728)  U~  as [16 token-groups][128 dv][4 tokens] fp32
 //   [73728, 73984)  e^{b_C - b_c} for c = 0..63, fp32 (rows past the chunk's length hold 1)

@@ -401,10 +401,10 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
     tc_fence_after_sync();
 
     const int d = (warp & 3) * 32 + (tid & 31);   // TMEM lane of this thread: a dk / dv index
-    {   // W^T[d][32 tokens] -> bf16 -> W image staged over the (now dead) K halves
+    {   // W^T[d][32 tokens] -> bf16 -> W image staged over the (now dead) K halves.  The image
+        // is MN-major for the state pass's product S W^T (one 128-byte row of 64 tokens per dk
+        // index), so a thread writes its own row in 16-byte pieces.
         uint8_t* sW = smem + kI_QK + 8192 + (d >> 6) * 16384;
-        const uint32_t wcol = ((d & 7) << 1);
-        const uint32_t wchunk = (d & 63) >> 3;
 #pragma unroll
         for (int step = 0; step < 2; ++step) {
             const int cbase = colhalf * 32 + step * 16;
@@ -412,9 +412,14 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
             tmem_ld16(tW + lane_base + cbase, x);
             tmem_wait_ld();
 #pragma unroll
-            for (int j = 0; j < 16; ++j)
-                *reinterpret_cast<__nv_bfloat16*>(sW + sw128_offset(cbase + j, wchunk) + wcol) =
-                    __float2bfloat16(__uint_as_float(x[j]));
+            for (int h = 0; h < 2; ++h) {
+                uint4 w;
+                w.x = pack_bf16(__uint_as_float(x[8 * h + 0]), __uint_as_float(x[8 * h + 1]));
+                w.y = pack_bf16(__uint_as_float(x[8 * h + 2]), __uint_as_float(x[8 * h + 3]));
+                w.z = pack_bf16(__uint_as_float(x[8 * h + 4]), __uint_as_float(x[8 * h + 5]));
+                w.w = pack_bf16(__uint_as_float(x[8 * h + 6]), __uint_as_float(x[8 * h + 7]));
+                *reinterpret_cast<uint4*>(sW + sw128_offset(d & 63, (cbase >> 3) + h)) = w;
+            }
         }
     }
     // the product that read T_w has retired: its place takes the remainder of T diag(beta)

@@ -144,12 +144,13 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
         if (lane == 0) {
             const uint32_t id64 = make_idesc_bf16(128, 64, false, false);
             const uint32_t id128mn = make_idesc_bf16(128, 128, false, true);
+            const uint32_t id64mn = make_idesc_bf16(128, 64, false, true);
             const uint32_t sRec0 = smem_u32(smem + kS_Rec), sRec1 = sRec0 + kStageBytes;
-            const uint64_t dW0 = make_sdesc_sw128(sRec0 + kRecW, 16, 1024);
+            const uint64_t dW0 = make_sdesc_sw128(sRec0 + kRecW, 8192, 1024);
             const uint64_t dQ0 = make_sdesc_sw128(sRec0 + kRecQg, 16, 1024);
             const uint64_t dP0 = make_sdesc_sw128(sRec0 + kRecP, 16, 1024);
             const uint64_t dK0 = make_sdesc_sw128(sRec0 + kS_K, 8192, 1024);
-            const uint64_t dW1 = make_sdesc_sw128(sRec1 + kRecW, 16, 1024);
+            const uint64_t dW1 = make_sdesc_sw128(sRec1 + kRecW, 8192, 1024);
             const uint64_t dQ1 = make_sdesc_sw128(sRec1 + kRecQg, 16, 1024);
             const uint64_t dP1 = make_sdesc_sw128(sRec1 + kRecP, 16, 1024);
             const uint64_t dK1 = make_sdesc_sw128(sRec1 + kS_K, 8192, 1024);
@@ -173,15 +174,15 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
                         break;
                     }
                     tc_fence_after_sync();
-                    // D1 = S W^T  (on the chain); k-step ks reads 16 dk: 32 bytes inside a half
-                    mma_ts_c<false>(tD1, tS, w, id64);
-                    mma_ts_c<true>(tD1, tS + 8, sdesc_advance(w, 32), id64);
-                    mma_ts_c<true>(tD1, tS + 16, sdesc_advance(w, 64), id64);
-                    mma_ts_c<true>(tD1, tS + 24, sdesc_advance(w, 96), id64);
-                    mma_ts_c<true>(tD1, tS + 32, sdesc_advance(w, 8192), id64);
-                    mma_ts_c<true>(tD1, tS + 40, sdesc_advance(w, 8192 + 32), id64);
-                    mma_ts_c<true>(tD1, tS + 48, sdesc_advance(w, 8192 + 64), id64);
-                    mma_ts_c<true>(tD1, tS + 56, sdesc_advance(w, 8192 + 96), id64);
+                    // D1 = S W^T  (on the chain); W is MN-major: k-step ks reads 16 dk rows = 2048 bytes
+                    mma_ts_c<false>(tD1, tS, w, id64mn);
+                    mma_ts_c<true>(tD1, tS + 8, sdesc_advance(w, 2048), id64mn);
+                    mma_ts_c<true>(tD1, tS + 16, sdesc_advance(w, 4096), id64mn);
+                    mma_ts_c<true>(tD1, tS + 24, sdesc_advance(w, 6144), id64mn);
+                    mma_ts_c<true>(tD1, tS + 32, sdesc_advance(w, 8192), id64mn);
+                    mma_ts_c<true>(tD1, tS + 40, sdesc_advance(w, 10240), id64mn);
+                    mma_ts_c<true>(tD1, tS + 48, sdesc_advance(w, 12288), id64mn);
+                    mma_ts_c<true>(tD1, tS + 56, sdesc_advance(w, 14336), id64mn);
                     mma_commit(&bar_d1);
                     // Y = S Qg^T  (off the chain)
                     mma_ts_c<false>(tY, tS, qg, id64);
