@@ -234,9 +234,8 @@ int gdn_prefill_fused(const void* q, const void* k, const void* v,
  * gdn_prefill_stream - the chunked algorithm in three launches whose state
  * pass is a persistent kernel: one CTA per SM walks a list of (sequence,
  * v-head) units and streams their chunks without draining its pipeline
- * between units.  It is the route for batches with many more units than SMs
- * (many short sequences).  Arguments, workspace and results are
- * gdn_prefill_chunked's.
+ * between units.  It is the route gdn_prefill takes for batches with more
+ * units than SMs.  Arguments, workspace and results are gdn_prefill_chunked's.
  */
 int gdn_prefill_stream(const void* q, const void* k, const void* v,
                        const float* g, const float* beta, const int32_t* cu_seqlens,

@@ -263,9 +263,10 @@ int gdn_prefill(const void* q, const void* k, const void* v, const float* g, con
     }
     const long long units = static_cast<long long>(N) * Hv;
     const bool few_units = units <= sms / 3 && longest > 16 * gdn::kChunk;
-    // Many more units than SMs (many short sequences): the persistent state pass, which does not
-    // pay a CTA start, a pipeline fill and a drain per unit.
-    const bool many_units = units >= 4LL * sms;
+    // More units than SMs: the persistent state pass, which does not pay a CTA start, a pipeline
+    // fill and a drain per unit (with at most one unit per SM the two state passes are equal and
+    // the plain one has the cheaper table-building launch).
+    const bool many_units = units > sms;
     const PrefillRoute route = coop && few_units ? kRouteFused : many_units ? kRouteStream : kRouteChunked;
     return prefill_chunked_impl(route, q, k, v, g, beta, cu_seqlens, init_state,
                                 final_state, slot_idx, o, T, N, Hqk, Hv, dk, dv, chunk, num_slots,

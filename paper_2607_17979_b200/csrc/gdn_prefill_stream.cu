@@ -17,8 +17,8 @@
 // that is two phases ahead), which is why the state hand-over after a unit's last chunk is
 // omitted rather than left unconsumed.
 //
-// The fp32 master state lives in TMEM as the accumulator of the state product, pre-scaled by the
-// next chunk's e^{b_C} (same scheme as the fused kernel's state role).
+// The fp32 master state lives in the epilogue threads' registers (64 per thread; TMEM lane = state
+// row, two column halves), as in the one-CTA-per-unit state kernel.
 #include "gdn_prefill_device.cuh"
 
 namespace gdn {
@@ -198,9 +198,8 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
                         break;
                     }
                     tc_fence_after_sync();
-                    // S_acc (= e^{b_C} S, prepared by the epilogue) += (U decayed, hi + lo) K
-                    // (K tile MN-major: 16 tokens = 2048 bytes)
-                    mma_ts_c<true>(tD4, tmem + kT_Us, kk, id128mn);
+                    // D4 = (U decayed, hi + lo) K   (K tile MN-major: 16 tokens = 2048 bytes)
+                    mma_ts_c<false>(tD4, tmem + kT_Us, kk, id128mn);
                     mma_ts_c<true>(tD4, tmem + kT_Us + 8, sdesc_advance(kk, 2048), id128mn);
                     mma_ts_c<true>(tD4, tmem + kT_Us + 16, sdesc_advance(kk, 4096), id128mn);
                     mma_ts_c<true>(tD4, tmem + kT_Us + 24, sdesc_advance(kk, 6144), id128mn);
@@ -229,17 +228,15 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
             __syncwarp();
             if (lane == 0) mbar_arrive(bar);
         };
-        const uint32_t tSacc = tmem + kT_D4 + lane_base + half * 64;     // this thread's 64 columns
-        const uint32_t tSbf = tmem + kT_S + lane_base + half * 32;
-        // 16 state columns at a time: fp32 values v[] -> bf16 copy, and gamma * v -> master
-        auto put_state = [&](const int c0, const float (&v)[16], const float gamma) {
-            uint32_t pk[8], sc[16];
+        float S[64];      // the thread's 64 state columns [64*half, 64*half+64) of row dv, fp32 master
+        auto store_state_bf16 = [&]() {           // S (fp32 regs) -> bf16 A operand in TMEM
 #pragma unroll
-            for (int i = 0; i < 8; ++i) pk[i] = pack_bf16(v[2 * i], v[2 * i + 1]);
+            for (int c0 = 0; c0 < 64; c0 += 32) {
+                uint32_t pk[16];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) sc[i] = __float_as_uint(gamma * v[i]);
-            tmem_st8(tSbf + (c0 >> 1), pk);
-            tmem_st16(tSacc + c0, sc);
+                for (int j = 0; j < 16; ++j) pk[j] = pack_bf16(S[c0 + 2 * j], S[c0 + 2 * j + 1]);
+                tmem_st16(tmem + kT_S + lane_base + half * 32 + (c0 >> 1), pk);
+            }
         };
         // The o rows of a chunk are produced one chunk later, in two parts that fit the two waits
         // of the chain: (A) scale, round, transpose into shared memory; (B) whole rows in 16-byte
@@ -308,24 +305,18 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
                 continue;
             }
             const int nc = u.nc;
-            // the unit's initial state: bf16 copy + master pre-scaled by chunk 0's e^{b_C}
-            await(&bar_full[gc & 1], (gc >> 1) & 1u);
-            if (ok) {
-                const float g0 = reinterpret_cast<const float*>(smem + (gc & 1) * kStageBytes + kS_Rec +
-                                                                kRecGammaC)[0];
-#pragma unroll 1
-                for (int c0 = 0; c0 < 64; c0 += 16) {
-                    float v[16];
+            // the unit's initial state
+            if (p.init_state) {
 #pragma unroll
-                    for (int i = 0; i < 16; i += 4) {
-                        const float4 x = p.init_state
-                                             ? *reinterpret_cast<const float4*>(p.init_state + tile_off + c0 + i)
-                                             : make_float4(0.f, 0.f, 0.f, 0.f);
-                        v[i] = x.x; v[i + 1] = x.y; v[i + 2] = x.z; v[i + 3] = x.w;
-                    }
-                    put_state(c0, v, g0);
+                for (int j = 0; j < 64; j += 4) {
+                    const float4 x = *reinterpret_cast<const float4*>(p.init_state + tile_off + j);
+                    S[j] = x.x; S[j + 1] = x.y; S[j + 2] = x.z; S[j + 3] = x.w;
                 }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 64; ++j) S[j] = 0.f;
             }
+            if (ok) store_state_bf16();
             hand_over(&bar_s);
             for (int j = 0; j < nc; ++j) {
                 const uint32_t g = gc + j;
@@ -381,28 +372,28 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
                 pend_len = min(kChunk, u.seq_len - j * kChunk);
                 pend_y = tmem + kT_Y + st * 64;
                 const bool last = j + 1 == nc;
-                if (!last) await(&bar_full[st ^ 1], ((g + 1) >> 1) & 1u);   // next record's e^{b_C}
                 await(&bar_d4, g & 1u);
-                if (ok) {   // the master now holds S(j+1): refresh the bf16 copy, pre-scale the master
-                    const float gn = last ? 1.f
-                                          : reinterpret_cast<const float*>(smem + (st ^ 1) * kStageBytes +
-                                                                           kS_Rec + kRecGammaC)[0];
-#pragma unroll 2
-                    for (int c0 = 0; c0 < 64; c0 += 16) {
-                        uint32_t x[16];
-                        tmem_ld16(tSacc + c0, x);
+                if (ok) {   // S <- e^{b_C} S + D4 on the thread's 64 dk columns
+                    const float gC = reinterpret_cast<const float*>(base + kS_Rec + kRecGammaC)[0];
+#pragma unroll
+                    for (int c0 = 0; c0 < 64; c0 += 32) {
+                        uint32_t xa[16], xb[16];
+                        tmem_ld16(tmem + kT_D4 + lane_base + half * 64 + c0, xa);
+                        tmem_ld16(tmem + kT_D4 + lane_base + half * 64 + c0 + 16, xb);
                         tmem_wait_ld();
-                        float v[16];
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(x[i]);
-                        if (!last) {
-                            put_state(c0, v, gn);
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < 16; i += 4)
-                                *reinterpret_cast<float4*>(p.final_state + tile_off + c0 + i) =
-                                    make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                        for (int jj = 0; jj < 16; ++jj) {
+                            S[c0 + jj] = fmaf(gC, S[c0 + jj], __uint_as_float(xa[jj]));
+                            S[c0 + 16 + jj] = fmaf(gC, S[c0 + 16 + jj], __uint_as_float(xb[jj]));
                         }
+                    }
+                    if (!last) {
+                        store_state_bf16();          // the next chunk's A operand
+                    } else {
+#pragma unroll
+                        for (int j4 = 0; j4 < 64; j4 += 4)
+                            *reinterpret_cast<float4*>(p.final_state + tile_off + j4) =
+                                make_float4(S[j4], S[j4 + 1], S[j4 + 2], S[j4 + 3]);
                     }
                 }
                 if (lane == 0) mbar_arrive(&bar_free[st]);     // this warp is done with the stage
