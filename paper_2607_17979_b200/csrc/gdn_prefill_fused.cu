@@ -180,6 +180,12 @@ __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
 __device__ __forceinline__ void st_release_u32(uint32_t* p, uint32_t v) {
     asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
+template <int kRegs> __device__ __forceinline__ void reg_alloc() {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegs));
+}
+template <int kRegs> __device__ __forceinline__ void reg_dealloc() {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegs));
+}
 __device__ __forceinline__ void fence_proxy_async_all() {
     asm volatile("fence.proxy.async;" ::: "memory");
 }
@@ -235,13 +241,16 @@ __device__ __forceinline__ void fused_intra_role(const TensorMaps& maps, const P
 }
 
 // ------------------------------------------------------------------ state role
-__device__ __forceinline__ void fused_state_role(const TensorMaps& maps, const PrefillParams& p,
-                                                 uint8_t* ws, const WorkspaceLayout& lay,
-                                                 uint8_t* smem, StateStatics& ss,
-                                                 const uint32_t tmem) {
+// kEpi = true: the copy the eight chain warps run; false: the issuing and loading warps' copy.
+// Two copies so that each is wholly dominated by its own register re-allocation (the compiler
+// budgets registers per setmaxnreg region).
+template <bool kEpi>
+__device__ __forceinline__ void fused_state_role_impl(const TensorMaps& maps, const PrefillParams& p,
+                                                      uint8_t* ws, const WorkspaceLayout& lay,
+                                                      uint8_t* smem, StateStatics& ss,
+                                                      const uint32_t tmem) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (warp > kFLoadWarp) return;                    // spare warps of the CTA
-    const bool is_epi = warp < kFEpiWarps;
+    constexpr bool is_epi = kEpi;
     const int half = (warp >> 2) & 1;                 // which half of the columns this thread owns
     const int dv = (warp & 3) * 32 + lane;            // TMEM lane = state row
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
@@ -329,7 +338,7 @@ __device__ __forceinline__ void fused_state_role(const TensorMaps& maps, const P
         auto par_chunk = [&](int j) { return (b_chunk + j) & 1u; };
         auto par_s = [&](int j) { return (b_s + j) & 1u; };
 
-        if (warp == kFLoadWarp) {
+        if (!kEpi && warp == kFLoadWarp) {
             // ===================== loading warp: wait for each record's flag, then copy it in
             if (lane == 0) {
                 const uint8_t* records =
@@ -363,7 +372,7 @@ __device__ __forceinline__ void fused_state_role(const TensorMaps& maps, const P
                 }
             }
             __syncwarp();
-        } else if (!is_epi) {
+        } else if constexpr (!kEpi) {
             // ===================== issuing warp: tensor-core instructions
             if (lane == 0) {
                 const uint32_t id64 = make_idesc_bf16(128, 64, false, false);
@@ -408,9 +417,8 @@ __device__ __forceinline__ void fused_state_role(const TensorMaps& maps, const P
                     mma_ts_c<true>(tY, tS + 56, sdesc_advance(qg, 8192 + 96), id64);
                     if (!wait_or_abort(&ss.bar_u, par_chunk(j), abortp)) break;    // U operands in TMEM
                     tc_fence_after_sync();
-                    // S_acc (= e^{b_C} S, prepared by the epilogue) += (U decayed, hi + lo) K
-                    // (K tile MN-major: 16 tokens = 2048 bytes)
-                    mma_ts_c<true>(tD4, tmem + kT_Us, kk, id128mn);
+                    // D4 = (U decayed, hi + lo) K   (K tile MN-major: 16 tokens = 2048 bytes)
+                    mma_ts_c<false>(tD4, tmem + kT_Us, kk, id128mn);
                     mma_ts_c<true>(tD4, tmem + kT_Us + 8, sdesc_advance(kk, 2048), id128mn);
                     mma_ts_c<true>(tD4, tmem + kT_Us + 16, sdesc_advance(kk, 4096), id128mn);
                     mma_ts_c<true>(tD4, tmem + kT_Us + 24, sdesc_advance(kk, 6144), id128mn);
@@ -431,26 +439,23 @@ __device__ __forceinline__ void fused_state_role(const TensorMaps& maps, const P
             __syncwarp();
         } else {
             // ===================== epilogue warps: U and the state refresh (the dependent chain)
-            // The fp32 master state lives in TMEM (tile kT_D4): before chunk j's state product it
-            // holds e^{b_C(j)} S(j), the product accumulates U^T K into it, and the refresh below
-            // turns the result S(j+1) into the bf16 operand copy and into e^{b_C(j+1)} S(j+1).
+            // The fp32 master state lives in registers (64 per thread: row dv, columns
+            // [64*half, 64*half + 64)); its bf16 copy in TMEM is the A operand of S W^T and S Qg^T.
             auto hand_over = [&](uint64_t* bar) {     // after tcgen05.st: publish to the issuing lane
                 tmem_wait_st();
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar);
             };
-            const uint32_t tSacc = tmem + kT_D4 + lane_base + half * 64;     // this thread's 64 columns
-            const uint32_t tSbf = tmem + kT_S + lane_base + half * 32;
-            // 16 state columns at a time: fp32 values v[] -> bf16 copy, and gamma * v -> master
-            auto put_state = [&](const int c0, const float (&v)[16], const float gamma) {
-                uint32_t pk[8], sc[16];
+            float S[64];
+            auto store_state_bf16 = [&]() {           // S (fp32 regs) -> bf16 A operand in TMEM
 #pragma unroll
-                for (int i = 0; i < 8; ++i) pk[i] = pack_bf16(v[2 * i], v[2 * i + 1]);
+                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    uint32_t pk[16];
 #pragma unroll
-                for (int i = 0; i < 16; ++i) sc[i] = __float_as_uint(gamma * v[i]);
-                tmem_st8(tSbf + (c0 >> 1), pk);
-                tmem_st16(tSacc + c0, sc);
+                    for (int j = 0; j < 16; ++j) pk[j] = pack_bf16(S[c0 + 2 * j], S[c0 + 2 * j + 1]);
+                    tmem_st16(tmem + kT_S + lane_base + half * 32 + (c0 >> 1), pk);
+                }
             };
             // o rows of chunk j from Y[j & 1] in two parts that fit the two waits of the chain:
             // (A) scale, round, transpose into shared memory; (B) whole rows in 16-byte pieces
@@ -490,22 +495,17 @@ __device__ __forceinline__ void fused_state_role(const TensorMaps& maps, const P
             // Every warp runs every group barrier and hand-over below, also after a wait has
             // failed (ok == false: later waits and all work are skipped), so that no warp is ever
             // left alone at a barrier.
-            await(&ss.bar_full[0], par_full(0));          // chunk 0's record: its e^{b_C} is needed
-            if (ok) {
-                const float g0 = reinterpret_cast<const float*>(smem + kS_Rec + kRecGammaC)[0];
-#pragma unroll 1
-                for (int c0 = 0; c0 < 64; c0 += 16) {
-                    float v[16];
+            if (p.init_state) {
 #pragma unroll
-                    for (int i = 0; i < 16; i += 4) {
-                        const float4 x = p.init_state
-                                             ? *reinterpret_cast<const float4*>(p.init_state + tile_off + c0 + i)
-                                             : make_float4(0.f, 0.f, 0.f, 0.f);
-                        v[i] = x.x; v[i + 1] = x.y; v[i + 2] = x.z; v[i + 3] = x.w;
-                    }
-                    put_state(c0, v, g0);
+                for (int j = 0; j < 64; j += 4) {
+                    const float4 x = *reinterpret_cast<const float4*>(p.init_state + tile_off + j);
+                    S[j] = x.x; S[j + 1] = x.y; S[j + 2] = x.z; S[j + 3] = x.w;
                 }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 64; ++j) S[j] = 0.f;
             }
+            store_state_bf16();
             hand_over(&ss.bar_s);
             for (int j = 0; j < nc; ++j) {
                 const int st = j & 1;
@@ -556,28 +556,28 @@ __device__ __forceinline__ void fused_state_role(const TensorMaps& maps, const P
                     if (ok) outputs_flush(j - 1);
                 }
                 const bool last = j + 1 == nc;
-                if (!last) await(&ss.bar_full[st ^ 1], par_full(j + 1));   // next record's e^{b_C}
                 await(&ss.bar_d4, par_chunk(j));
-                if (ok) {   // the master now holds S(j+1): refresh the bf16 copy, pre-scale the master
-                    const float gn = last ? 1.f
-                                          : reinterpret_cast<const float*>(smem + (st ^ 1) * kStageBytes +
-                                                                           kS_Rec + kRecGammaC)[0];
-#pragma unroll 2
-                    for (int c0 = 0; c0 < 64; c0 += 16) {
-                        uint32_t x[16];
-                        tmem_ld16(tSacc + c0, x);
+                if (ok) {   // S <- e^{b_C} S + D4 on the thread's 64 dk columns
+                    const float gC = reinterpret_cast<const float*>(base + kS_Rec + kRecGammaC)[0];
+#pragma unroll
+                    for (int c0 = 0; c0 < 64; c0 += 32) {
+                        uint32_t xa[16], xb[16];
+                        tmem_ld16(tmem + kT_D4 + lane_base + half * 64 + c0, xa);
+                        tmem_ld16(tmem + kT_D4 + lane_base + half * 64 + c0 + 16, xb);
                         tmem_wait_ld();
-                        float v[16];
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(x[i]);
-                        if (!last) {
-                            put_state(c0, v, gn);
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < 16; i += 4)
-                                *reinterpret_cast<float4*>(p.final_state + tile_off + c0 + i) =
-                                    make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                        for (int jj = 0; jj < 16; ++jj) {
+                            S[c0 + jj] = fmaf(gC, S[c0 + jj], __uint_as_float(xa[jj]));
+                            S[c0 + 16 + jj] = fmaf(gC, S[c0 + 16 + jj], __uint_as_float(xb[jj]));
                         }
+                    }
+                    if (!last) {
+                        store_state_bf16();
+                    } else {
+#pragma unroll
+                        for (int j4 = 0; j4 < 64; j4 += 4)
+                            *reinterpret_cast<float4*>(p.final_state + tile_off + j4) =
+                                make_float4(S[j4], S[j4 + 1], S[j4 + 2], S[j4 + 3]);
                     }
                 }
                 if (lane == 0) mbar_arrive(&ss.bar_free[st]);     // this warp is done with the stage
@@ -597,6 +597,26 @@ __device__ __forceinline__ void fused_state_role(const TensorMaps& maps, const P
             mbar_wait(&ss.bar_full[0], 0, 1u << 12);
             mbar_wait(&ss.bar_full[1], 0, 1u << 12);
         }
+    }
+}
+
+__device__ __forceinline__ void fused_state_role(const TensorMaps& maps, const PrefillParams& p,
+                                                 uint8_t* ws, const WorkspaceLayout& lay,
+                                                 uint8_t* smem, StateStatics& ss,
+                                                 const uint32_t tmem) {
+    // The kernel is compiled for 768 threads (80 registers each) because of the producer CTAs.
+    // In a state-pass CTA the fourteen spare warps and the issuing / loading warps hand most of
+    // their registers back and the eight chain warps take 168 each, enough to keep the fp32
+    // master state in registers (setmaxnreg works on groups of four warps).
+    const int warp = threadIdx.x >> 5;
+    if (warp >= 12) {
+        reg_dealloc<24>();                            // spare warps of the CTA
+    } else if (warp >= 8) {
+        reg_dealloc<64>();
+        if (warp <= kFLoadWarp) fused_state_role_impl<false>(maps, p, ws, lay, smem, ss, tmem);
+    } else {
+        reg_alloc<168>();
+        fused_state_role_impl<true>(maps, p, ws, lay, smem, ss, tmem);
     }
 }
 
