@@ -263,10 +263,10 @@ int gdn_prefill(const void* q, const void* k, const void* v, const float* g, con
     }
     const long long units = static_cast<long long>(N) * Hv;
     const bool few_units = units <= sms / 3 && longest > 16 * gdn::kChunk;
-    // More units than SMs: the persistent state pass, which does not pay a CTA start, a pipeline
-    // fill and a drain per unit (with at most one unit per SM the two state passes are equal and
-    // the plain one has the cheaper table-building launch).
-    const bool many_units = units > sms;
+    // The persistent state pass does not pay a CTA start, a pipeline fill and a drain per unit and
+    // its loader is a warp of its own; measured equal or faster from about half a unit per SM
+    // up.  Below that the plain pass has the cheaper table-building launch.
+    const bool many_units = 2 * units > sms;
     const PrefillRoute route = coop && few_units ? kRouteFused : many_units ? kRouteStream : kRouteChunked;
     return prefill_chunked_impl(route, q, k, v, g, beta, cu_seqlens, init_state,
                                 final_state, slot_idx, o, T, N, Hqk, Hv, dk, dv, chunk, num_slots,

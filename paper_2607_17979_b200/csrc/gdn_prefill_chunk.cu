@@ -19,6 +19,7 @@ prefill_prep_kernel(const int32_t* __restrict__ cu, int32_t T, int32_t N, uint8_
     __shared__ int32_t warp_sums[kPrepThreads / 32];
     __shared__ int32_t running;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    pdl_launch_dependents();        // the next kernel's CTAs may become resident (they wait for us)
     if (tid == 0) {
         running = 0;
         if (cu[0] != 0 || cu[N] != T) report(dev_status, kDevBadCuSeqlens);
@@ -76,6 +77,8 @@ prefill_intra_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
                      const WorkspaceLayout lay) {
     const int c = blockIdx.x;
     const int hv = blockIdx.y;
+    pdl_launch_dependents();
+    pdl_wait();                     // the chunk table is the previous kernel's
     const int32_t total = *reinterpret_cast<const int32_t*>(ws);
     if (c >= total) return;
     const ChunkInfo ci = reinterpret_cast<const ChunkInfo*>(ws + lay.chunks)[c];
@@ -126,6 +129,7 @@ prefill_state_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
 
     const int32_t* seq_first = reinterpret_cast<const int32_t*>(ws + lay.seq_first);
     const int32_t* seq_bad = reinterpret_cast<const int32_t*>(ws + lay.seq_bad);
+    pdl_wait();                     // tables and records are the previous kernels'
     if (seq_bad[n]) return;
     const int c_first = seq_first[n];
     const int nc = seq_first[n + 1] - c_first;
@@ -483,8 +487,8 @@ cudaError_t launch_prefill_intra(const TensorMaps& maps, const ChunkedParams& cp
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kIntraSmem);
     if (e != cudaSuccess) return e;
     dim3 grid(cp.lay.max_chunks, cp.p.Hv);
-    prefill_intra_kernel<<<grid, kIntraThreads, kIntraSmem, stream>>>(maps, cp.p, cp.ws, cp.lay);
-    return cudaGetLastError();
+    return launch_dependent(prefill_intra_kernel, grid, dim3(kIntraThreads), kIntraSmem, stream, maps,
+                            cp.p, cp.ws, cp.lay);
 }
 
 cudaError_t launch_prefill_chunked(const ChunkedParams& cp, cudaStream_t stream) {
@@ -503,8 +507,8 @@ cudaError_t launch_prefill_chunked(const ChunkedParams& cp, cudaStream_t stream)
         e = launch_prefill_intra(maps, cp, stream);
         if (e != cudaSuccess) return e;
     }
-    prefill_state_kernel<<<p.N * p.Hv, kStateThreads, kStateSmem, stream>>>(maps, p, cp.ws, cp.lay);
-    return cudaGetLastError();
+    return launch_dependent(prefill_state_kernel, dim3(p.N * p.Hv), dim3(kStateThreads), kStateSmem,
+                            stream, maps, p, cp.ws, cp.lay);
 }
 
 }  // namespace gdn

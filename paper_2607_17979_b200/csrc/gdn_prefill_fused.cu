@@ -35,6 +35,7 @@ prefill_fused_prep_kernel(const int32_t* __restrict__ cu, int32_t T, int32_t N, 
     __shared__ int32_t warp_sums[kFPrepThreads / 32];
     __shared__ int32_t running;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    pdl_launch_dependents();        // the next kernel's CTAs may become resident (they wait for us)
 
     for (int i = tid; i < lay.max_nc + 2; i += kFPrepThreads) { hist[i] = 0; fill[i] = 0; }
     for (size_t i = tid; i < static_cast<size_t>(lay.max_chunks) * Hv; i += kFPrepThreads) flags[i] = 0u;

@@ -99,6 +99,7 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
     tc_fence_after_sync();
     const uint32_t tmem = tmem_base_s;
     volatile int* abortp = &abort_flag;
+    pdl_wait();                     // tables and records are the previous kernels'
 
     // gc = chunks of earlier units of this CTA; chunk j of the current unit is chunk g = gc + j of
     // the CTA's stream: stage g & 1, phase g >> 1 of bar_full / bar_free of that stage, phase g of
@@ -443,8 +444,8 @@ cudaError_t launch_prefill_stream(const ChunkedParams& cp, cudaStream_t stream) 
     }
     const long long units = static_cast<long long>(p.N) * p.Hv;
     const int grid = static_cast<int>(units < sms ? units : sms);
-    prefill_state_stream_kernel<<<grid, kStreamThreads, kStreamSmem, stream>>>(maps, p, cp.ws, cp.lay);
-    return cudaGetLastError();
+    return launch_dependent(prefill_state_stream_kernel, dim3(grid), dim3(kStreamThreads), kStreamSmem,
+                            stream, maps, p, cp.ws, cp.lay);
 }
 
 }  // namespace gdn
