@@ -105,7 +105,8 @@ cudaError_t launch_prefill_fused(const ChunkedParams& cp, cudaStream_t stream);
 // stream their records without draining between units (for batches with many more units than SMs).
 cudaError_t launch_prefill_stream(const ChunkedParams& cp, cudaStream_t stream);
 // Pieces shared by the launchers: the prep kernel that also ranks the sequences by chunk count
-// (longest first) and clears the queues and flags; the intra-chunk kernel over all items.
-cudaError_t launch_prefill_ranked_prep(const ChunkedParams& cp, cudaStream_t stream);
+// (longest first) and, for the fused launch, orders the chunks and clears the queues and flags;
+// the intra-chunk kernel over all items.
+cudaError_t launch_prefill_ranked_prep(const ChunkedParams& cp, cudaStream_t stream, bool for_fused);
 
 }  // namespace gdn

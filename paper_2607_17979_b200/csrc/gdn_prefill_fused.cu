@@ -20,7 +20,8 @@ constexpr int kFPrepThreads = 256;
 
 __global__ void __launch_bounds__(kFPrepThreads)
 prefill_fused_prep_kernel(const int32_t* __restrict__ cu, int32_t T, int32_t N, int32_t Hv,
-                          uint8_t* ws, WorkspaceLayout lay, int32_t* dev_status) {
+                          uint8_t* ws, WorkspaceLayout lay, int32_t* dev_status,
+                          const int for_fused) {   // 0: only the chunk table and the ranking
     int32_t* hdr = reinterpret_cast<int32_t*>(ws);
     int32_t* seq_first = reinterpret_cast<int32_t*>(ws + lay.seq_first);
     int32_t* seq_bad = reinterpret_cast<int32_t*>(ws + lay.seq_bad);
@@ -38,7 +39,9 @@ prefill_fused_prep_kernel(const int32_t* __restrict__ cu, int32_t T, int32_t N, 
     pdl_launch_dependents();        // the next kernel's CTAs may become resident (they wait for us)
 
     for (int i = tid; i < lay.max_nc + 2; i += kFPrepThreads) { hist[i] = 0; fill[i] = 0; }
-    for (size_t i = tid; i < static_cast<size_t>(lay.max_chunks) * Hv; i += kFPrepThreads) flags[i] = 0u;
+    if (for_fused)
+        for (size_t i = tid; i < static_cast<size_t>(lay.max_chunks) * Hv; i += kFPrepThreads)
+            flags[i] = 0u;
     if (tid == 0) {
         running = 0;
         hdr[kHdrItemHead] = 0;
@@ -116,8 +119,8 @@ prefill_fused_prep_kernel(const int32_t* __restrict__ cu, int32_t T, int32_t N, 
     }
     if (tid == 0) running = 0;
     __syncthreads();
-    // pos[j] = number of chunks at positions < j: exclusive prefix sum of cnt
-    for (int base = 0; base <= lay.max_nc; base += kFPrepThreads) {
+    // pos[j] = number of chunks at positions < j: exclusive prefix sum of cnt (fused launch only)
+    for (int base = 0; for_fused && base <= lay.max_nc; base += kFPrepThreads) {
         const int j = base + tid;
         const int32_t x = j <= lay.max_nc ? cnt[j] : 0;
         int32_t incl = x;
@@ -143,7 +146,8 @@ prefill_fused_prep_kernel(const int32_t* __restrict__ cu, int32_t T, int32_t N, 
         const int32_t rank = cnt[nc] + atomicAdd(&fill[nc], 1);
         seq_by_rank[rank] = n;
         const int32_t first = seq_first[n];
-        for (int j = 0; j < nc; ++j) order[pos[j] + rank] = first + j;
+        if (for_fused)
+            for (int j = 0; j < nc; ++j) order[pos[j] + rank] = first + j;
     }
 }
 
@@ -653,10 +657,10 @@ prefill_fused_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
 // =============================================================================================
 // host side
 // =============================================================================================
-cudaError_t launch_prefill_ranked_prep(const ChunkedParams& cp, cudaStream_t stream) {
+cudaError_t launch_prefill_ranked_prep(const ChunkedParams& cp, cudaStream_t stream, bool for_fused) {
     prefill_fused_prep_kernel<<<1, kFPrepThreads, 0, stream>>>(cp.p.cu_seqlens, cp.p.T, cp.p.N,
                                                                cp.p.Hv, cp.ws, cp.lay,
-                                                               cp.p.dev_status);
+                                                               cp.p.dev_status, for_fused ? 1 : 0);
     return cudaGetLastError();
 }
 
@@ -674,7 +678,7 @@ cudaError_t launch_prefill_fused(const ChunkedParams& cp, cudaStream_t stream) {
     TensorMaps maps;
     if (!make_prefill_tensor_maps(&maps, p)) return cudaErrorInvalidValue;
 
-    e = launch_prefill_ranked_prep(cp, stream);
+    e = launch_prefill_ranked_prep(cp, stream, true);
     if (e != cudaSuccess) return e;
 
     // How many CTAs run the state pass: measured best near 0.43 of the SMs when there are more

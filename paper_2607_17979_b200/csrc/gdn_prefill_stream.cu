@@ -436,7 +436,7 @@ cudaError_t launch_prefill_stream(const ChunkedParams& cp, cudaStream_t stream) 
     if (e != cudaSuccess) return e;
     TensorMaps maps;
     if (!make_prefill_tensor_maps(&maps, p)) return cudaErrorInvalidValue;
-    e = launch_prefill_ranked_prep(cp, stream);
+    e = launch_prefill_ranked_prep(cp, stream, false);
     if (e != cudaSuccess) return e;
     if (cp.lay.max_chunks > 0) {
         e = launch_prefill_intra(maps, cp, stream);
