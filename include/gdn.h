@@ -198,10 +198,13 @@ int gdn_prefill(const void* q, const void* k, const void* v,
                 int32_t* dev_status, void* stream);
 
 /*
- * gdn_prefill routes by the longest sequence: at most GDN_RECURRENT_MAX_SEQLEN
- * tokens (by max_seqlen_hint if given, else by the bound T) goes to the
- * token-by-token kernel, anything longer to the chunked kernels.  The two
- * routes below can also be called directly; arguments are gdn_prefill's.
+ * gdn_prefill routes by shape: a batch whose longest sequence has at most
+ * GDN_RECURRENT_MAX_SEQLEN tokens (by max_seqlen_hint if given, else by the
+ * bound T) goes to the token-by-token kernel; anything longer to one of the
+ * chunked variants (gdn_prefill_fused for a few long sequence-heads,
+ * gdn_prefill_stream from about half a sequence-head per SM up, else
+ * gdn_prefill_chunked).  Each route can also be called directly; arguments
+ * are gdn_prefill's.
  */
 #define GDN_RECURRENT_MAX_SEQLEN 16
 int gdn_prefill_chunked(const void* q, const void* k, const void* v,
@@ -216,7 +219,7 @@ int gdn_prefill_chunked(const void* q, const void* k, const void* v,
 
 /*
  * gdn_prefill_fused - the chunked algorithm in one cooperative launch (plus a
- * small table-building launch): a third of the SMs walk the sequences' chunks
+ * small table-building launch): some of the SMs walk the sequences' chunks
  * in order while the others produce the per-chunk quantities just ahead of
  * them.  Arguments, workspace and results are gdn_prefill_chunked's.
  */

@@ -1,8 +1,8 @@
 // Chunked prefill in ONE cooperative launch: the record producers and the state pass overlap.
 //
 // The grid has one CTA of 768 threads per SM.  The first `n_state` CTAs run the serial state pass
-// (16 epilogue warps + 1 issuing warp), each pulling (sequence, v-head) units from a queue,
-// longest sequence first.  The other CTAs run three independent groups of 256 threads that pull
+// (8 chain warps + an issuing warp + a loading warp), each pulling (sequence, v-head) units from
+// a queue, longest sequence first.  The other CTAs run three independent groups of 256 threads that pull
 // (chunk, v-head) items from a second queue and write their records (the intra-chunk routine of
 // gdn_prefill_device.cuh), in the order the state pass consumes them: by position inside the
 // sequence first, by sequence rank second.  A record is published through a flag in global
@@ -279,7 +279,7 @@ __device__ __forceinline__ void fused_state_role_impl(const TensorMaps& maps, co
     if (tid == 0) {
         mbar_init(&ss.bar_full[0], 1);
         mbar_init(&ss.bar_full[1], 1);
-        mbar_init(&ss.bar_free[0], kFEpiWarps + 1);     // 16 epilogue warps + the last product
+        mbar_init(&ss.bar_free[0], kFEpiWarps + 1);     // the chain warps + the last product
         mbar_init(&ss.bar_free[1], kFEpiWarps + 1);
         mbar_init(&ss.bar_d1, 1);
         mbar_init(&ss.bar_d4, 1);
