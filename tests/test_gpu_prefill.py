@@ -157,29 +157,67 @@ def test_chunked_and_recurrent_routes_agree():
 
 
 def test_prefill_varlen_benchmark_config_full():
-    """4 sequences {512,1024,2048,4096}, 32 v-heads: every output against the oracle."""
+    """4 sequences {512,1024,2048,4096}, 32 v-heads: every output against the oracle, through the
+    length-routed entry point (the call the benchmark times) and through the plain three launches."""
     p = I.make_config(3, 0)
-    o, S, o_ref, S_ref = compare(p, "chunked")
-    U.check_state(S.astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
+    o_ref, S_ref, _ = oracle_prefill(p)
     cu = p["cu_seqlens"]
-    for n in range(4):                                               # no sequence hides in the norm
-        U.check_o(o[cu[n]:cu[n + 1]], o_ref[cu[n]:cu[n + 1]], U.O_REL_L2_PREFILL)
+    for impl in ("auto", "chunked"):
+        o, S, status = run_prefill(p, impl)
+        assert status == 0
+        U.check_o(o, o_ref, U.O_REL_L2_PREFILL)
+        U.check_state(S.astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
+        for n in range(4):                                           # no sequence hides in the norm
+            U.check_o(o[cu[n]:cu[n + 1]], o_ref[cu[n]:cu[n + 1]], U.O_REL_L2_PREFILL)
 
 
 def test_prefill_long_context_benchmark_config_sampled_heads():
-    """One 32768-token sequence at full size on the GPU; the oracle recomputes four sampled
-    v-heads (each with its own q/k head) over the whole sequence."""
+    """One 32768-token sequence at full size on the GPU, through the length-routed entry point
+    (the fused launch for this shape) and the plain three launches; the oracle recomputes four
+    sampled v-heads (each with its own q/k head) over the whole sequence."""
     p = I.make_config(4, 0)
-    o, S, status = run_prefill(p, "chunked")
-    assert status == 0 and np.isfinite(o).all() and np.isfinite(S).all()
+    refs = {}
     for hv in (0, 13, 22, 31):
         hq = hv // 2
-        o_ref, S_ref, _ = oracle.prefill(p["q"][:, hq:hq + 1], p["k"][:, hq:hq + 1], p["v"][:, hv:hv + 1],
-                                         p["g"][:, hv:hv + 1], p["beta"][:, hv:hv + 1], p["cu_seqlens"],
-                                         p["init_state"][:, hv:hv + 1].astype(np.float64), None, p["scale"])
-        U.check_o(o[:, hv:hv + 1], o_ref, U.O_REL_L2_PREFILL)
-        U.check_o(o[-4096:, hv:hv + 1], o_ref[-4096:], U.O_REL_L2_PREFILL)   # the far end of the carry
-        U.check_state(S[:, hv:hv + 1].astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
+        refs[hv] = oracle.prefill(p["q"][:, hq:hq + 1], p["k"][:, hq:hq + 1], p["v"][:, hv:hv + 1],
+                                  p["g"][:, hv:hv + 1], p["beta"][:, hv:hv + 1], p["cu_seqlens"],
+                                  p["init_state"][:, hv:hv + 1].astype(np.float64), None, p["scale"])
+    for impl in ("auto", "chunked"):
+        o, S, status = run_prefill(p, impl)
+        assert status == 0 and np.isfinite(o).all() and np.isfinite(S).all()
+        for hv, (o_ref, S_ref, _) in refs.items():
+            U.check_o(o[:, hv:hv + 1], o_ref, U.O_REL_L2_PREFILL)
+            U.check_o(o[-4096:, hv:hv + 1], o_ref[-4096:], U.O_REL_L2_PREFILL)   # the far end of the carry
+            U.check_state(S[:, hv:hv + 1].astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
+
+
+@pytest.mark.parametrize("impl", ["auto", "chunked", "stream", "fused"])
+def test_batches_that_are_all_padding_or_all_empty(impl):
+    """No valid work at all: every slot negative (rows zeroed, no state touched), and every
+    sequence but one empty (states pass through bit-exactly)."""
+    p = I.prefill_inputs([70, 5, 130], 2, 4, seed=31, init="normal")
+    slots = np.array([-1, -5, -2], np.int32)
+    o, S, status = run_prefill(p, impl, slot_idx=slots, pool_fill=3.0)
+    assert status == 0
+    assert np.array_equal(o, np.zeros_like(o)) and np.array_equal(S, np.full_like(S, 3.0))
+    q = I.prefill_inputs([0, 0, 90, 0], 2, 4, seed=32, init="normal")
+    o, S, o_ref, S_ref = compare(q, impl)
+    assert np.array_equal(S[[0, 1, 3]], q["init_state"][[0, 1, 3]])
+    U.check_state(S[2:3].astype(np.float64), S_ref[2:3], U.STATE_REL_L2_PREFILL)
+
+
+def test_thousands_of_tiny_sequences():
+    """2000 sequences of 1-40 tokens, 4 v-heads (8000 units): the length-routed entry point and
+    the persistent state pass against the oracle."""
+    rng = np.random.default_rng(11)
+    lens = [int(x) for x in rng.integers(1, 41, size=2000)]
+    p = I.prefill_inputs(lens, 2, 4, seed=33, init="normal")
+    o_ref, S_ref, _ = oracle_prefill(p)
+    for impl in ("auto", "stream"):
+        o, S, status = run_prefill(p, impl)
+        assert status == 0
+        U.check_o(o, o_ref, U.O_REL_L2_PREFILL)
+        U.check_state(S.astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
 
 
 def test_chunked_repeatable_under_load_many_ctas():
