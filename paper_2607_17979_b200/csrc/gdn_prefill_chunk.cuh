@@ -14,7 +14,9 @@
 // intra-chunk kernel (one CTA per chunk and v-head, all chunks in parallel)
 // computes W, U~, P and b with tcgen05 GEMMs and an fp32 triangular solve and
 // writes them as a record; the state-pass kernel (one CTA per sequence and
-// v-head) walks the chunks in order carrying S in fp32 registers.
+// v-head, or one persistent CTA per SM walking a list of them) walks the chunks
+// in order carrying S in fp32 registers.  A fused variant runs the last two as
+// one cooperative launch.
 #pragma once
 #include "gdn_common.cuh"
 #include <cuda.h>
