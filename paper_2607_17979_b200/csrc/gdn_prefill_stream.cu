@@ -68,7 +68,8 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                                ~static_cast<uintptr_t>(1023));
-    __shared__ uint64_t bar_full[2], bar_free[2], bar_d1, bar_d4, bar_y, bar_s, bar_u;
+    __shared__ uint64_t bar_full[2], bar_free_a[2], bar_free_b[2], bar_free_c[2], bar_d1, bar_d4, bar_y,
+        bar_s, bar_u;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_flag;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -80,8 +81,16 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
     if (tid == 0) {
         mbar_init(&bar_full[0], 1);
         mbar_init(&bar_full[1], 1);
-        mbar_init(&bar_free[0], kSEpiWarps + 1);     // the epilogue warps + the chunk's last product
-        mbar_init(&bar_free[1], kSEpiWarps + 1);
+        // A stage is released in three parts as its readers finish with them, so that the next
+        // record's copies start up to half a chunk step earlier (one chunk step of look-ahead is
+        // shorter than a cold 74 KB copy): W and Qg once S W^T and S Qg^T have retired, U~ and the
+        // decay vector once every chain warp has read them, P and the K tile once U P^T and the
+        // state product have retired.
+        for (int st = 0; st < 2; ++st) {
+            mbar_init(&bar_free_a[st], 1);
+            mbar_init(&bar_free_b[st], kSEpiWarps);
+            mbar_init(&bar_free_c[st], 1);
+        }
         mbar_init(&bar_d1, 1);
         mbar_init(&bar_d4, 1);
         mbar_init(&bar_y, 1);
@@ -102,7 +111,7 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
     pdl_wait();                     // tables and records are the previous kernels'
 
     // gc = chunks of earlier units of this CTA; chunk j of the current unit is chunk g = gc + j of
-    // the CTA's stream: stage g & 1, phase g >> 1 of bar_full / bar_free of that stage, phase g of
+    // the CTA's stream: stage g & 1, phase g >> 1 of bar_full / bar_free_* of that stage, phase g of
     // bar_d1 / bar_d4 / bar_y / bar_u and of bar_s (one state hand-over per chunk: the initial one
     // and one after every chunk but the unit's last).
     uint32_t gc = 0;
@@ -123,15 +132,17 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
                 for (int j = 0; j < u.nc; ++j) {
                     const uint32_t g = gc + j;
                     const int st = g & 1;
-                    // the stage held chunk g - 2: free once that chunk's last product has retired
-                    // and every epilogue warp is done with its record
-                    if (g >= 2 && !wait_or_abort(&bar_free[st], ((g - 2) >> 1) & 1u, abortp)) {
-                        live = false;
-                        break;
-                    }
+                    // the stage held chunk g - 2; each part is refilled as soon as it is free
+                    const uint32_t par_free = ((g - 2) >> 1) & 1u;
                     uint8_t* base = smem + st * kStageBytes;
+                    const uint8_t* rec = records + j * rec_stride;
+                    if (g >= 2 && !wait_or_abort(&bar_free_a[st], par_free, abortp)) { live = false; break; }
                     mbar_expect_tx(&bar_full[st], kRecBytes + 16384);
-                    bulk_load(base + kS_Rec, records + j * rec_stride, kRecBytes, &bar_full[st]);
+                    bulk_load(base + kS_Rec + kRecW, rec + kRecW, kRecP - kRecW, &bar_full[st]);
+                    if (g >= 2 && !wait_or_abort(&bar_free_b[st], par_free, abortp)) { live = false; break; }
+                    bulk_load(base + kS_Rec + kRecU, rec + kRecU, kRecBytes - kRecU, &bar_full[st]);
+                    if (g >= 2 && !wait_or_abort(&bar_free_c[st], par_free, abortp)) { live = false; break; }
+                    bulk_load(base + kS_Rec + kRecP, rec + kRecP, kRecU - kRecP, &bar_full[st]);
                     tma_load_2d(base + kS_K, &maps.k, u.hqk * kD, u.seq_t0 + j * kChunk, &bar_full[st]);
                     tma_load_2d(base + kS_K + 8192, &maps.k, u.hqk * kD + 64, u.seq_t0 + j * kChunk,
                                 &bar_full[st]);
@@ -194,6 +205,7 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
                     mma_ts_c<true>(tY, tS + 40, sdesc_advance(qg, 8192 + 32), id64);
                     mma_ts_c<true>(tY, tS + 48, sdesc_advance(qg, 8192 + 64), id64);
                     mma_ts_c<true>(tY, tS + 56, sdesc_advance(qg, 8192 + 96), id64);
+                    mma_commit(&bar_free_a[st]);                          // W and Qg have been read
                     if (!wait_or_abort(&bar_u, g & 1u, abortp)) {         // U operands in TMEM
                         live = false;
                         break;
@@ -215,7 +227,7 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
                     mma_ts_c<true>(tY, tmem + kT_U + 16, sdesc_advance(pp, 64), id64);
                     mma_ts_c<true>(tY, tmem + kT_U + 24, sdesc_advance(pp, 96), id64);
                     mma_commit(&bar_y);
-                    mma_commit(&bar_free[st]);
+                    mma_commit(&bar_free_c[st]);                          // P and the K tile have been read
                 }
                 gc += u.nc;
             }
@@ -363,7 +375,9 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
                         tmem_st8(tmem + kT_U + lane_base + (cb >> 1), pu);
                     }
                 }
+                const float gC = reinterpret_cast<const float*>(base + kS_Rec + kRecGammaC)[0];
                 hand_over(&bar_u);
+                if (lane == 0) mbar_arrive(&bar_free_b[st]);    // this warp has read U~, decay, e^{b_C}
                 if (pend) {     // part B, while this chunk's state product is in flight
                     epi_group_sync();
                     if (ok) outputs_flush();
@@ -375,7 +389,6 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
                 const bool last = j + 1 == nc;
                 await(&bar_d4, g & 1u);
                 if (ok) {   // S <- e^{b_C} S + D4 on the thread's 64 dk columns
-                    const float gC = reinterpret_cast<const float*>(base + kS_Rec + kRecGammaC)[0];
 #pragma unroll
                     for (int c0 = 0; c0 < 64; c0 += 32) {
                         uint32_t xa[16], xb[16];
@@ -397,7 +410,6 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
                                 make_float4(S[j4], S[j4 + 1], S[j4 + 2], S[j4 + 3]);
                     }
                 }
-                if (lane == 0) mbar_arrive(&bar_free[st]);     // this warp is done with the stage
                 if (!last) hand_over(&bar_s);
             }
             gc += nc;
