@@ -5,12 +5,17 @@
 // The one-CTA-per-unit state kernel pays, for every unit, a launch slot, barrier and TMEM set-up,
 // the first record's memory latency and the tail of its last chunk; with thousands of short
 // units (many short sequences) that overhead is longer than the chunk steps themselves.  Here
-//   * warp 9 (loader) copies records and K tiles in unit order, running up to two chunks ahead
+//   * warp 13 (loader) copies records and K tiles in unit order, running up to two chunks ahead
 //     of the consumers and straight across unit boundaries;
-//   * warp 8 (issuer) issues every tcgen05.mma;
-//   * warps 0-7 (epilogue) carry the dependent chain  D1 = S W^T -> U = U~ - D1 ->
-//     S_acc += (U decayed)^T K -> refresh, and turn Y = S Qg^T + U P^T into o rows.
-// The three roles never meet at a CTA barrier inside the loop: each derives the same unit list
+//   * warp 12 (issuer) issues every tcgen05.mma;
+//   * warps 0-7 (chain) carry the dependent chain  D1 = S W^T -> U = U~ - D1 ->
+//     D4 = (U decayed)^T K -> S = e^{b_C} S + D4 and nothing else;
+//   * warps 8-11 (output) turn Y = S Qg^T + U P^T into o rows one chunk behind, so that no
+//     output work sits in the chain warps' instruction stream (it cost about 500 of the 4300
+//     cycles of a chunk step there).
+// The CTA is compiled for 512 threads (128 registers); the chain warps take 168 registers each
+// from what the other groups hand back (setmaxnreg).
+// The roles never meet at a CTA barrier inside the loop: each derives the same unit list
 // (unit = blockIdx.x + i * gridDim.x over the rank-sorted units, longest sequences first) and the
 // same running chunk count, from which every mbarrier parity follows.  Every barrier phase is
 // consumed by its waiter before the next one can complete (a parity wait cannot tell a barrier
@@ -23,11 +28,13 @@
 
 namespace gdn {
 
-constexpr int kSEpiWarps = 8;
+constexpr int kSEpiWarps = 8;                 // warps 0-7: the dependent chain
 constexpr int kSEpiThreads = kSEpiWarps * 32;
-constexpr int kSIssueWarp = kSEpiWarps;
-constexpr int kSLoadWarp = kSEpiWarps + 1;
-constexpr int kStreamThreads = kSEpiThreads + 64;
+constexpr int kSOutWarp0 = 8;                 // warps 8-11: output rows (one per TMEM lane quadrant)
+constexpr int kSOutThreads = 128;
+constexpr int kSIssueWarp = 12;               // warp 12: tcgen05.mma issue
+constexpr int kSLoadWarp = 13;                // warp 13: record and K-tile copies (14, 15 spare)
+constexpr int kStreamThreads = 512;
 constexpr uint32_t kStreamSmem = 2 * kStageBytes + 16384 + 1024;
 
 namespace {
@@ -68,8 +75,8 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                                ~static_cast<uintptr_t>(1023));
-    __shared__ uint64_t bar_full[2], bar_free_a[2], bar_free_b[2], bar_free_c[2], bar_d1, bar_d4, bar_y,
-        bar_s, bar_u;
+    __shared__ uint64_t bar_full[2], bar_free_a[2], bar_free_b[2], bar_free_c[2], bar_yfree[2], bar_y[2],
+        bar_d1, bar_d4, bar_s, bar_u;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_flag;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -90,10 +97,12 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
             mbar_init(&bar_free_a[st], 1);
             mbar_init(&bar_free_b[st], kSEpiWarps);
             mbar_init(&bar_free_c[st], 1);
+            mbar_init(&bar_yfree[st], kSOutThreads / 32);   // the output warps have read the tile
         }
         mbar_init(&bar_d1, 1);
         mbar_init(&bar_d4, 1);
-        mbar_init(&bar_y, 1);
+        mbar_init(&bar_y[0], 1);      // one per Y tile: with a single barrier the output warps could
+        mbar_init(&bar_y[1], 1);      // find it two phases ahead, which a parity wait cannot tell
         mbar_init(&bar_s, kSEpiWarps);
         mbar_init(&bar_u, kSEpiWarps);
         abort_flag = 0;
@@ -116,6 +125,8 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
     // and one after every chunk but the unit's last).
     uint32_t gc = 0;
 
+    if (warp >= kSIssueWarp) {
+    reg_dealloc<56>();
     if (warp == kSLoadWarp) {
         // ===================== loader: records and K tiles, in stream order
         if (lane == 0) {
@@ -196,7 +207,11 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
                     mma_ts_c<true>(tD1, tS + 48, sdesc_advance(w, 12288), id64mn);
                     mma_ts_c<true>(tD1, tS + 56, sdesc_advance(w, 14336), id64mn);
                     mma_commit(&bar_d1);
-                    // Y = S Qg^T  (off the chain)
+                    // Y = S Qg^T  (off the chain) overwrites the tile the output warps read two chunks ago
+                    if (g >= 2 && !wait_or_abort(&bar_yfree[st], ((g - 2) >> 1) & 1u, abortp)) {
+                        live = false;
+                        break;
+                    }
                     mma_ts_c<false>(tY, tS, qg, id64);
                     mma_ts_c<true>(tY, tS + 8, sdesc_advance(qg, 32), id64);
                     mma_ts_c<true>(tY, tS + 16, sdesc_advance(qg, 64), id64);
@@ -226,15 +241,17 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
                     mma_ts_c<true>(tY, tmem + kT_U + 8, sdesc_advance(pp, 32), id64);
                     mma_ts_c<true>(tY, tmem + kT_U + 16, sdesc_advance(pp, 64), id64);
                     mma_ts_c<true>(tY, tmem + kT_U + 24, sdesc_advance(pp, 96), id64);
-                    mma_commit(&bar_y);
+                    mma_commit(&bar_y[st]);
                     mma_commit(&bar_free_c[st]);                          // P and the K tile have been read
                 }
                 gc += u.nc;
             }
         }
         __syncwarp();
-    } else {
-        // ===================== epilogue warps: U, the state refresh (the dependent chain), o rows
+    }
+    } else if (warp < kSEpiWarps) {
+        reg_alloc<168>();
+        // ===================== chain warps: U and the state refresh (the dependent chain)
         auto hand_over = [&](uint64_t* bar) {     // after tcgen05.st: publish to the issuing lane
             tmem_wait_st();
             tc_fence_before_sync();
@@ -251,39 +268,6 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
                 tmem_st16(tmem + kT_S + lane_base + half * 32 + (c0 >> 1), pk);
             }
         };
-        // The o rows of a chunk are produced one chunk later, in two parts that fit the two waits
-        // of the chain: (A) scale, round, transpose into shared memory; (B) whole rows in 16-byte
-        // pieces.  `pend_*` describe the chunk whose rows are still owed (it may belong to the
-        // previous unit).
-        bool pend = false;
-        __nv_bfloat16* pend_og = nullptr;
-        int pend_len = 0;
-        uint32_t pend_y = 0;
-        const size_t tok_stride = static_cast<size_t>(p.Hv) * kD;
-        auto outputs_stage = [&]() {
-            __nv_bfloat16* sO = reinterpret_cast<__nv_bfloat16*>(smem + kS_Out);
-#pragma unroll
-            for (int c0 = 0; c0 < 32; c0 += 16) {
-                uint32_t x[16];
-                tmem_ld16(pend_y + lane_base + half * 32 + c0, x);
-                tmem_wait_ld();
-#pragma unroll
-                for (int jj = 0; jj < 16; ++jj)
-                    sO[(half * 32 + c0 + jj) * kD + dv] =
-                        __float2bfloat16(p.scale * __uint_as_float(x[jj]));
-            }
-        };
-        auto outputs_flush = [&]() {
-            const __nv_bfloat16* sO = reinterpret_cast<const __nv_bfloat16*>(smem + kS_Out);
-#pragma unroll
-            for (int it = 0; it < 4; ++it) {
-                const int row = it * 16 + (tid >> 4), piece = tid & 15;
-                if (row < pend_len)
-                    *reinterpret_cast<uint4*>(pend_og + row * tok_stride + piece * 8) =
-                        *reinterpret_cast<const uint4*>(sO + row * kD + piece * 8);
-            }
-        };
-
         bool ok = true;
         auto await = [&](uint64_t* bar, uint32_t parity) {   // bounded wait + tcgen05 fence
             if (ok && !warp_wait_or_abort(bar, parity, abortp)) ok = false;
@@ -335,11 +319,6 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
                 const uint32_t g = gc + j;
                 const int st = g & 1;
                 const uint8_t* base = smem + st * kStageBytes;
-                if (pend) {     // part A of the previous chunk's rows, while D1 is in flight
-                    await(&bar_y, (g - 1) & 1u);
-                    epi_group_sync();
-                    if (ok) outputs_stage();
-                }
                 await(&bar_full[st], (g >> 1) & 1u);
                 await(&bar_d1, g & 1u);
                 if (ok) {   // U^T[dv][c] = U~^T - D1 for the thread's 32 tokens [32*half, 32*half+32)
@@ -378,14 +357,6 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
                 const float gC = reinterpret_cast<const float*>(base + kS_Rec + kRecGammaC)[0];
                 hand_over(&bar_u);
                 if (lane == 0) mbar_arrive(&bar_free_b[st]);    // this warp has read U~, decay, e^{b_C}
-                if (pend) {     // part B, while this chunk's state product is in flight
-                    epi_group_sync();
-                    if (ok) outputs_flush();
-                }
-                pend = true;
-                pend_og = p.o + (static_cast<size_t>(u.seq_t0 + j * kChunk) * p.Hv + u.hv) * kD;
-                pend_len = min(kChunk, u.seq_len - j * kChunk);
-                pend_y = tmem + kT_Y + st * 64;
                 const bool last = j + 1 == nc;
                 await(&bar_d4, g & 1u);
                 if (ok) {   // S <- e^{b_C} S + D4 on the thread's 64 dk columns
@@ -414,12 +385,60 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
             }
             gc += nc;
         }
-        if (pend) {     // the rows of the stream's last chunk
-            await(&bar_y, (gc - 1) & 1u);
-            epi_group_sync();
-            if (ok) outputs_stage();
-            epi_group_sync();
-            if (ok) outputs_flush();
+    } else {
+        reg_dealloc<80>();
+        // ===================== output warps: Y = S Qg^T + U P^T (fp32, TMEM) -> o rows.  Warp 8 + q
+        // reads TMEM lanes 32 q .. 32 q + 31 (dv indices), scales and rounds, transposes through
+        // shared memory, and the four warps write whole rows in 16-byte pieces.
+        const int q4 = warp & 3;
+        const int odv = q4 * 32 + lane;
+        const uint32_t olane = static_cast<uint32_t>(q4 * 32) << 16;
+        const int ot = tid - kSOutWarp0 * 32;
+        const size_t tok_stride = static_cast<size_t>(p.Hv) * kD;
+        __nv_bfloat16* sO = reinterpret_cast<__nv_bfloat16*>(smem + kS_Out);
+        auto out_sync = [] { asm volatile("bar.sync 1, %0;" ::"n"(kSOutThreads) : "memory"); };
+        bool ok = true;
+        UnitInfo nxt = unit_info(p, ws, lay, min(static_cast<int>(blockIdx.x), total_units - 1));
+        for (int unit = blockIdx.x; unit < total_units; unit += gridDim.x) {
+            const UnitInfo u = nxt;
+            nxt = unit_info(p, ws, lay, min(unit + static_cast<int>(gridDim.x), total_units - 1));
+            if (u.skip) continue;
+            for (int j = 0; j < u.nc; ++j) {
+                const uint32_t g = gc + j;
+                const int buf = g & 1;
+                // every warp runs both group barriers of every chunk, also after a failed wait
+                if (ok && !warp_wait_or_abort(&bar_y[buf], (g >> 1) & 1u, abortp)) ok = false;
+                tc_fence_after_sync();
+                if (ok) {
+                    const uint32_t tY = tmem + kT_Y + buf * 64;
+#pragma unroll
+                    for (int c0 = 0; c0 < 64; c0 += 16) {
+                        uint32_t x[16];
+                        tmem_ld16(tY + olane + c0, x);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int jj = 0; jj < 16; ++jj)
+                            sO[(c0 + jj) * kD + odv] = __float2bfloat16(p.scale * __uint_as_float(x[jj]));
+                    }
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bar_yfree[buf]);     // the tile may be overwritten
+                out_sync();
+                if (ok) {
+                    const int len = min(kChunk, u.seq_len - j * kChunk);
+                    __nv_bfloat16* og = p.o + (static_cast<size_t>(u.seq_t0 + j * kChunk) * p.Hv + u.hv) * kD;
+#pragma unroll
+                    for (int it = 0; it < 8; ++it) {
+                        const int row = it * 8 + (ot >> 4), piece = ot & 15;
+                        if (row < len)
+                            *reinterpret_cast<uint4*>(og + row * tok_stride + piece * 8) =
+                                *reinterpret_cast<const uint4*>(sO + row * kD + piece * 8);
+                    }
+                }
+                out_sync();
+            }
+            gc += u.nc;
         }
     }
 

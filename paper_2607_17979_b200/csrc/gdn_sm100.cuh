@@ -239,6 +239,17 @@ __device__ __forceinline__ uint32_t sw128_offset(uint32_t row, uint32_t chunk) {
     return row * 128u + ((chunk ^ (row & 7u)) << 4);
 }
 
+// Register re-allocation between the warp groups (four consecutive warps) of a CTA: a group that
+// needs few registers hands the rest back, another takes them.  The compiler budgets registers
+// per region only for code that the instruction dominates, so each role's code must sit wholly
+// behind its own call.
+template <int kRegs> __device__ __forceinline__ void reg_alloc() {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegs));
+}
+template <int kRegs> __device__ __forceinline__ void reg_dealloc() {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegs));
+}
+
 // Programmatic dependent launch: a kernel launched with the programmatic-stream-serialization
 // attribute may start while its predecessor in the stream is still running; it must not touch
 // the predecessor's results before pdl_wait() (a no-op under an ordinary launch).  The
