@@ -164,7 +164,7 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
         __syncwarp();
     } else if (warp == kSIssueWarp) {
         // ===================== issuer: tensor-core instructions
-        if (lane == 0) {
+        {   // the whole warp runs this warp-uniform code; one elected lane executes each tcgen05 instruction
             const uint32_t id64 = make_idesc_bf16(128, 64, false, false);
             const uint32_t id128mn = make_idesc_bf16(128, 128, false, true);
             const uint32_t id64mn = make_idesc_bf16(128, 64, false, true);
@@ -198,51 +198,51 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
                     }
                     tc_fence_after_sync();
                     // D1 = S W^T  (on the chain); W is MN-major: k-step ks reads 16 dk rows = 2048 bytes
-                    mma_ts_c<false>(tD1, tS, w, id64mn);
-                    mma_ts_c<true>(tD1, tS + 8, sdesc_advance(w, 2048), id64mn);
-                    mma_ts_c<true>(tD1, tS + 16, sdesc_advance(w, 4096), id64mn);
-                    mma_ts_c<true>(tD1, tS + 24, sdesc_advance(w, 6144), id64mn);
-                    mma_ts_c<true>(tD1, tS + 32, sdesc_advance(w, 8192), id64mn);
-                    mma_ts_c<true>(tD1, tS + 40, sdesc_advance(w, 10240), id64mn);
-                    mma_ts_c<true>(tD1, tS + 48, sdesc_advance(w, 12288), id64mn);
-                    mma_ts_c<true>(tD1, tS + 56, sdesc_advance(w, 14336), id64mn);
-                    mma_commit(&bar_d1);
+                    if (elect_one()) mma_ts_c<false>(tD1, tS, w, id64mn);
+                    if (elect_one()) mma_ts_c<true>(tD1, tS + 8, sdesc_advance(w, 2048), id64mn);
+                    if (elect_one()) mma_ts_c<true>(tD1, tS + 16, sdesc_advance(w, 4096), id64mn);
+                    if (elect_one()) mma_ts_c<true>(tD1, tS + 24, sdesc_advance(w, 6144), id64mn);
+                    if (elect_one()) mma_ts_c<true>(tD1, tS + 32, sdesc_advance(w, 8192), id64mn);
+                    if (elect_one()) mma_ts_c<true>(tD1, tS + 40, sdesc_advance(w, 10240), id64mn);
+                    if (elect_one()) mma_ts_c<true>(tD1, tS + 48, sdesc_advance(w, 12288), id64mn);
+                    if (elect_one()) mma_ts_c<true>(tD1, tS + 56, sdesc_advance(w, 14336), id64mn);
+                    if (elect_one()) mma_commit(&bar_d1);
                     // Y = S Qg^T  (off the chain) overwrites the tile the output warps read two chunks ago
                     if (g >= 2 && !wait_or_abort(&bar_yfree[st], ((g - 2) >> 1) & 1u, abortp)) {
                         live = false;
                         break;
                     }
-                    mma_ts_c<false>(tY, tS, qg, id64);
-                    mma_ts_c<true>(tY, tS + 8, sdesc_advance(qg, 32), id64);
-                    mma_ts_c<true>(tY, tS + 16, sdesc_advance(qg, 64), id64);
-                    mma_ts_c<true>(tY, tS + 24, sdesc_advance(qg, 96), id64);
-                    mma_ts_c<true>(tY, tS + 32, sdesc_advance(qg, 8192), id64);
-                    mma_ts_c<true>(tY, tS + 40, sdesc_advance(qg, 8192 + 32), id64);
-                    mma_ts_c<true>(tY, tS + 48, sdesc_advance(qg, 8192 + 64), id64);
-                    mma_ts_c<true>(tY, tS + 56, sdesc_advance(qg, 8192 + 96), id64);
-                    mma_commit(&bar_free_a[st]);                          // W and Qg have been read
+                    if (elect_one()) mma_ts_c<false>(tY, tS, qg, id64);
+                    if (elect_one()) mma_ts_c<true>(tY, tS + 8, sdesc_advance(qg, 32), id64);
+                    if (elect_one()) mma_ts_c<true>(tY, tS + 16, sdesc_advance(qg, 64), id64);
+                    if (elect_one()) mma_ts_c<true>(tY, tS + 24, sdesc_advance(qg, 96), id64);
+                    if (elect_one()) mma_ts_c<true>(tY, tS + 32, sdesc_advance(qg, 8192), id64);
+                    if (elect_one()) mma_ts_c<true>(tY, tS + 40, sdesc_advance(qg, 8192 + 32), id64);
+                    if (elect_one()) mma_ts_c<true>(tY, tS + 48, sdesc_advance(qg, 8192 + 64), id64);
+                    if (elect_one()) mma_ts_c<true>(tY, tS + 56, sdesc_advance(qg, 8192 + 96), id64);
+                    if (elect_one()) mma_commit(&bar_free_a[st]);                          // W and Qg have been read
                     if (!wait_or_abort(&bar_u, g & 1u, abortp)) {         // U operands in TMEM
                         live = false;
                         break;
                     }
                     tc_fence_after_sync();
                     // D4 = (U decayed, hi + lo) K   (K tile MN-major: 16 tokens = 2048 bytes)
-                    mma_ts_c<false>(tD4, tmem + kT_Us, kk, id128mn);
-                    mma_ts_c<true>(tD4, tmem + kT_Us + 8, sdesc_advance(kk, 2048), id128mn);
-                    mma_ts_c<true>(tD4, tmem + kT_Us + 16, sdesc_advance(kk, 4096), id128mn);
-                    mma_ts_c<true>(tD4, tmem + kT_Us + 24, sdesc_advance(kk, 6144), id128mn);
-                    mma_ts_c<true>(tD4, tmem + kT_UsLo, kk, id128mn);
-                    mma_ts_c<true>(tD4, tmem + kT_UsLo + 8, sdesc_advance(kk, 2048), id128mn);
-                    mma_ts_c<true>(tD4, tmem + kT_UsLo + 16, sdesc_advance(kk, 4096), id128mn);
-                    mma_ts_c<true>(tD4, tmem + kT_UsLo + 24, sdesc_advance(kk, 6144), id128mn);
-                    mma_commit(&bar_d4);
+                    if (elect_one()) mma_ts_c<false>(tD4, tmem + kT_Us, kk, id128mn);
+                    if (elect_one()) mma_ts_c<true>(tD4, tmem + kT_Us + 8, sdesc_advance(kk, 2048), id128mn);
+                    if (elect_one()) mma_ts_c<true>(tD4, tmem + kT_Us + 16, sdesc_advance(kk, 4096), id128mn);
+                    if (elect_one()) mma_ts_c<true>(tD4, tmem + kT_Us + 24, sdesc_advance(kk, 6144), id128mn);
+                    if (elect_one()) mma_ts_c<true>(tD4, tmem + kT_UsLo, kk, id128mn);
+                    if (elect_one()) mma_ts_c<true>(tD4, tmem + kT_UsLo + 8, sdesc_advance(kk, 2048), id128mn);
+                    if (elect_one()) mma_ts_c<true>(tD4, tmem + kT_UsLo + 16, sdesc_advance(kk, 4096), id128mn);
+                    if (elect_one()) mma_ts_c<true>(tD4, tmem + kT_UsLo + 24, sdesc_advance(kk, 6144), id128mn);
+                    if (elect_one()) mma_commit(&bar_d4);
                     // Y += U P^T
-                    mma_ts_c<true>(tY, tmem + kT_U, pp, id64);
-                    mma_ts_c<true>(tY, tmem + kT_U + 8, sdesc_advance(pp, 32), id64);
-                    mma_ts_c<true>(tY, tmem + kT_U + 16, sdesc_advance(pp, 64), id64);
-                    mma_ts_c<true>(tY, tmem + kT_U + 24, sdesc_advance(pp, 96), id64);
-                    mma_commit(&bar_y[st]);
-                    mma_commit(&bar_free_c[st]);                          // P and the K tile have been read
+                    if (elect_one()) mma_ts_c<true>(tY, tmem + kT_U, pp, id64);
+                    if (elect_one()) mma_ts_c<true>(tY, tmem + kT_U + 8, sdesc_advance(pp, 32), id64);
+                    if (elect_one()) mma_ts_c<true>(tY, tmem + kT_U + 16, sdesc_advance(pp, 64), id64);
+                    if (elect_one()) mma_ts_c<true>(tY, tmem + kT_U + 24, sdesc_advance(pp, 96), id64);
+                    if (elect_one()) mma_commit(&bar_y[st]);
+                    if (elect_one()) mma_commit(&bar_free_c[st]);                          // P and the K tile have been read
                 }
                 gc += u.nc;
             }
