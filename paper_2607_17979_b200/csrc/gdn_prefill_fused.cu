@@ -161,14 +161,16 @@ constexpr int kFEpiWarps = 8;                        // state role: warps 0-7 ch
 constexpr int kFEpiThreads = kFEpiWarps * 32;
 constexpr int kFIssueWarp = kFEpiWarps;              //   warp 8: tcgen05.mma issue
 constexpr int kFLoadWarp = kFEpiWarps + 1;           //   warp 9: record flags and TMA copies
-constexpr int kFRoleThreads = kFEpiThreads + 64;     // threads that take part in the state role
+constexpr int kFOutWarp0 = 12;                       //   warps 12-15: output rows
+constexpr int kFOutThreads = 128;
+constexpr int kFRoleThreads = kFEpiThreads + 64 + kFOutThreads;   // threads that take part in the state role
 constexpr uint32_t kFStateSmem = 2 * kStageBytes + 16384;
 constexpr uint32_t kFusedSmem =
     (kFGroups * kFGroupSmem > kFStateSmem ? kFGroups * kFGroupSmem : kFStateSmem) + 1024;
 constexpr uint32_t kSpinFlagLimit = 1u << 22;
 
 struct StateStatics {
-    uint64_t bar_full[2], bar_free[2], bar_d1, bar_d4, bar_y, bar_s, bar_u;
+    uint64_t bar_full[2], bar_free[2], bar_y[2], bar_yfree[2], bar_d1, bar_d4, bar_s, bar_u;
     int unit;
     int abort_flag;
 };
@@ -240,15 +242,16 @@ __device__ __forceinline__ void fused_intra_role(const TensorMaps& maps, const P
 }
 
 // ------------------------------------------------------------------ state role
-// kEpi = true: the copy the eight chain warps run; false: the issuing and loading warps' copy.
-// Two copies so that each is wholly dominated by its own register re-allocation (the compiler
-// budgets registers per setmaxnreg region).
-template <bool kEpi>
+// kRole 1: the copy the eight chain warps run; 0: the issuing and loading warps' copy; 2: the four
+// output warps' copy.  One copy per register budget, so that each is wholly dominated by its own
+// register re-allocation (the compiler budgets registers per setmaxnreg region).
+template <int kRole>
 __device__ __forceinline__ void fused_state_role_impl(const TensorMaps& maps, const PrefillParams& p,
                                                       uint8_t* ws, const WorkspaceLayout& lay,
                                                       uint8_t* smem, StateStatics& ss,
                                                       const uint32_t tmem) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    constexpr bool kEpi = kRole == 1, kOut = kRole == 2, kIssueLoad = kRole == 0;
     constexpr bool is_epi = kEpi;
     const int half = (warp >> 2) & 1;                 // which half of the columns this thread owns
     const int dv = (warp & 3) * 32 + lane;            // TMEM lane = state row
@@ -262,7 +265,7 @@ __device__ __forceinline__ void fused_state_role_impl(const TensorMaps& maps, co
     const int G = p.Hv / p.Hqk;
     volatile int* abortp = &ss.abort_flag;
     auto role_sync = [] { named_sync<4, kFRoleThreads>(); };
-    auto epi_sync = [] { named_sync<5, kFEpiThreads>(); };
+    auto out_sync = [] { named_sync<5, kFOutThreads>(); };
 
     // The mbarriers are initialised once and keep flipping phase from unit to unit (an mbarrier
     // must not be re-initialised while it is a valid object).  Every role thread keeps the same
@@ -277,7 +280,10 @@ __device__ __forceinline__ void fused_state_role_impl(const TensorMaps& maps, co
         mbar_init(&ss.bar_free[1], kFEpiWarps + 1);
         mbar_init(&ss.bar_d1, 1);
         mbar_init(&ss.bar_d4, 1);
-        mbar_init(&ss.bar_y, 1);
+        mbar_init(&ss.bar_y[0], 1);                    // one per Y tile, see the persistent pass
+        mbar_init(&ss.bar_y[1], 1);
+        mbar_init(&ss.bar_yfree[0], kFOutThreads / 32);
+        mbar_init(&ss.bar_yfree[1], kFOutThreads / 32);
         mbar_init(&ss.bar_s, kFEpiWarps);
         mbar_init(&ss.bar_u, kFEpiWarps);
         fence_barrier_init();
@@ -305,7 +311,7 @@ __device__ __forceinline__ void fused_state_role_impl(const TensorMaps& maps, co
             if (!seq_bad[n]) {
                 if (slot >= p.num_slots && tid == 0) report(p.dev_status, kDevBadSlot);
                 const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-                for (int idx = tid; idx < seq_len * 16; idx += kFRoleThreads)
+                for (int idx = tid; is_epi && idx < seq_len * 16; idx += kFEpiThreads)
                     *reinterpret_cast<uint4*>(p.o + (static_cast<size_t>(seq_t0 + (idx >> 4)) * p.Hv + hv) * kD +
                                               (idx & 15) * 8) = zero;
             }
@@ -337,7 +343,7 @@ __device__ __forceinline__ void fused_state_role_impl(const TensorMaps& maps, co
         auto par_chunk = [&](int j) { return (b_chunk + j) & 1u; };
         auto par_s = [&](int j) { return (b_s + j) & 1u; };
 
-        if (!kEpi && warp == kFLoadWarp) {
+        if (kIssueLoad && warp == kFLoadWarp) {
             // ===================== loading warp: wait for each record's flag, then copy it in
             if (lane == 0) {
                 const uint8_t* records =
@@ -371,9 +377,10 @@ __device__ __forceinline__ void fused_state_role_impl(const TensorMaps& maps, co
                 }
             }
             __syncwarp();
-        } else if constexpr (!kEpi) {
+        } else if constexpr (kIssueLoad) {
             // ===================== issuing warp: tensor-core instructions
-            if (lane == 0) {
+            // (warp-uniform code run by the whole warp; one elected lane executes each instruction)
+            {
                 const uint32_t id64 = make_idesc_bf16(128, 64, false, false);
                 const uint32_t id128mn = make_idesc_bf16(128, 128, false, true);
                 const uint32_t id64mn = make_idesc_bf16(128, 64, false, true);
@@ -396,48 +403,93 @@ __device__ __forceinline__ void fused_state_role_impl(const TensorMaps& maps, co
                     if (!wait_or_abort(&ss.bar_s, par_s(j), abortp)) break;    // bf16 S of chunk j in TMEM
                     tc_fence_after_sync();
                     // D1 = S W^T  (on the chain); W is MN-major: k-step ks reads 16 dk rows = 2048 bytes
-                    mma_ts_c<false>(tD1, tS, w, id64mn);
-                    mma_ts_c<true>(tD1, tS + 8, sdesc_advance(w, 2048), id64mn);
-                    mma_ts_c<true>(tD1, tS + 16, sdesc_advance(w, 4096), id64mn);
-                    mma_ts_c<true>(tD1, tS + 24, sdesc_advance(w, 6144), id64mn);
-                    mma_ts_c<true>(tD1, tS + 32, sdesc_advance(w, 8192), id64mn);
-                    mma_ts_c<true>(tD1, tS + 40, sdesc_advance(w, 10240), id64mn);
-                    mma_ts_c<true>(tD1, tS + 48, sdesc_advance(w, 12288), id64mn);
-                    mma_ts_c<true>(tD1, tS + 56, sdesc_advance(w, 14336), id64mn);
-                    mma_commit(&ss.bar_d1);
-                    // Y = S Qg^T  (off the chain)
-                    mma_ts_c<false>(tY, tS, qg, id64);
-                    mma_ts_c<true>(tY, tS + 8, sdesc_advance(qg, 32), id64);
-                    mma_ts_c<true>(tY, tS + 16, sdesc_advance(qg, 64), id64);
-                    mma_ts_c<true>(tY, tS + 24, sdesc_advance(qg, 96), id64);
-                    mma_ts_c<true>(tY, tS + 32, sdesc_advance(qg, 8192), id64);
-                    mma_ts_c<true>(tY, tS + 40, sdesc_advance(qg, 8192 + 32), id64);
-                    mma_ts_c<true>(tY, tS + 48, sdesc_advance(qg, 8192 + 64), id64);
-                    mma_ts_c<true>(tY, tS + 56, sdesc_advance(qg, 8192 + 96), id64);
+                    if (elect_one()) mma_ts_c<false>(tD1, tS, w, id64mn);
+                    if (elect_one()) mma_ts_c<true>(tD1, tS + 8, sdesc_advance(w, 2048), id64mn);
+                    if (elect_one()) mma_ts_c<true>(tD1, tS + 16, sdesc_advance(w, 4096), id64mn);
+                    if (elect_one()) mma_ts_c<true>(tD1, tS + 24, sdesc_advance(w, 6144), id64mn);
+                    if (elect_one()) mma_ts_c<true>(tD1, tS + 32, sdesc_advance(w, 8192), id64mn);
+                    if (elect_one()) mma_ts_c<true>(tD1, tS + 40, sdesc_advance(w, 10240), id64mn);
+                    if (elect_one()) mma_ts_c<true>(tD1, tS + 48, sdesc_advance(w, 12288), id64mn);
+                    if (elect_one()) mma_ts_c<true>(tD1, tS + 56, sdesc_advance(w, 14336), id64mn);
+                    if (elect_one()) mma_commit(&ss.bar_d1);
+                    // Y = S Qg^T  (off the chain) overwrites the tile the output warps read two chunks ago
+                    if (j >= 2 && !wait_or_abort(&ss.bar_yfree[st], par_full(j - 2), abortp)) break;
+                    if (elect_one()) mma_ts_c<false>(tY, tS, qg, id64);
+                    if (elect_one()) mma_ts_c<true>(tY, tS + 8, sdesc_advance(qg, 32), id64);
+                    if (elect_one()) mma_ts_c<true>(tY, tS + 16, sdesc_advance(qg, 64), id64);
+                    if (elect_one()) mma_ts_c<true>(tY, tS + 24, sdesc_advance(qg, 96), id64);
+                    if (elect_one()) mma_ts_c<true>(tY, tS + 32, sdesc_advance(qg, 8192), id64);
+                    if (elect_one()) mma_ts_c<true>(tY, tS + 40, sdesc_advance(qg, 8192 + 32), id64);
+                    if (elect_one()) mma_ts_c<true>(tY, tS + 48, sdesc_advance(qg, 8192 + 64), id64);
+                    if (elect_one()) mma_ts_c<true>(tY, tS + 56, sdesc_advance(qg, 8192 + 96), id64);
                     if (!wait_or_abort(&ss.bar_u, par_chunk(j), abortp)) break;    // U operands in TMEM
                     tc_fence_after_sync();
                     // D4 = (U decayed, hi + lo) K   (K tile MN-major: 16 tokens = 2048 bytes)
-                    mma_ts_c<false>(tD4, tmem + kT_Us, kk, id128mn);
-                    mma_ts_c<true>(tD4, tmem + kT_Us + 8, sdesc_advance(kk, 2048), id128mn);
-                    mma_ts_c<true>(tD4, tmem + kT_Us + 16, sdesc_advance(kk, 4096), id128mn);
-                    mma_ts_c<true>(tD4, tmem + kT_Us + 24, sdesc_advance(kk, 6144), id128mn);
-                    mma_ts_c<true>(tD4, tmem + kT_UsLo, kk, id128mn);
-                    mma_ts_c<true>(tD4, tmem + kT_UsLo + 8, sdesc_advance(kk, 2048), id128mn);
-                    mma_ts_c<true>(tD4, tmem + kT_UsLo + 16, sdesc_advance(kk, 4096), id128mn);
-                    mma_ts_c<true>(tD4, tmem + kT_UsLo + 24, sdesc_advance(kk, 6144), id128mn);
-                    mma_commit(&ss.bar_d4);
+                    if (elect_one()) mma_ts_c<false>(tD4, tmem + kT_Us, kk, id128mn);
+                    if (elect_one()) mma_ts_c<true>(tD4, tmem + kT_Us + 8, sdesc_advance(kk, 2048), id128mn);
+                    if (elect_one()) mma_ts_c<true>(tD4, tmem + kT_Us + 16, sdesc_advance(kk, 4096), id128mn);
+                    if (elect_one()) mma_ts_c<true>(tD4, tmem + kT_Us + 24, sdesc_advance(kk, 6144), id128mn);
+                    if (elect_one()) mma_ts_c<true>(tD4, tmem + kT_UsLo, kk, id128mn);
+                    if (elect_one()) mma_ts_c<true>(tD4, tmem + kT_UsLo + 8, sdesc_advance(kk, 2048), id128mn);
+                    if (elect_one()) mma_ts_c<true>(tD4, tmem + kT_UsLo + 16, sdesc_advance(kk, 4096), id128mn);
+                    if (elect_one()) mma_ts_c<true>(tD4, tmem + kT_UsLo + 24, sdesc_advance(kk, 6144), id128mn);
+                    if (elect_one()) mma_commit(&ss.bar_d4);
                     // Y += U P^T
-                    mma_ts_c<true>(tY, tmem + kT_U, pp, id64);
-                    mma_ts_c<true>(tY, tmem + kT_U + 8, sdesc_advance(pp, 32), id64);
-                    mma_ts_c<true>(tY, tmem + kT_U + 16, sdesc_advance(pp, 64), id64);
-                    mma_ts_c<true>(tY, tmem + kT_U + 24, sdesc_advance(pp, 96), id64);
-                    mma_commit(&ss.bar_y);
-                    mma_commit(&ss.bar_free[st]);
+                    if (elect_one()) mma_ts_c<true>(tY, tmem + kT_U, pp, id64);
+                    if (elect_one()) mma_ts_c<true>(tY, tmem + kT_U + 8, sdesc_advance(pp, 32), id64);
+                    if (elect_one()) mma_ts_c<true>(tY, tmem + kT_U + 16, sdesc_advance(pp, 64), id64);
+                    if (elect_one()) mma_ts_c<true>(tY, tmem + kT_U + 24, sdesc_advance(pp, 96), id64);
+                    if (elect_one()) mma_commit(&ss.bar_y[st]);
+                    if (elect_one()) mma_commit(&ss.bar_free[st]);
                 }
             }
             __syncwarp();
+        } else if constexpr (kOut) {
+            // ===================== output warps: Y = S Qg^T + U P^T (fp32, TMEM) -> o rows, one warp
+            // per TMEM lane quadrant; transposed through shared memory, written as whole rows
+            const int q4 = warp & 3;
+            const int odv = q4 * 32 + lane;
+            const uint32_t olane = static_cast<uint32_t>(q4 * 32) << 16;
+            const int ot = tid - kFOutWarp0 * 32;
+            const size_t tok_stride = static_cast<size_t>(p.Hv) * kD;
+            __nv_bfloat16* sO = reinterpret_cast<__nv_bfloat16*>(smem + kS_Out);
+            bool ok = true;
+            for (int j = 0; j < nc; ++j) {
+                const int buf = j & 1;
+                // every warp runs both group barriers of every chunk, also after a failed wait
+                if (ok && !warp_wait_or_abort(&ss.bar_y[buf], par_full(j), abortp)) ok = false;
+                tc_fence_after_sync();
+                if (ok) {
+                    const uint32_t tY = tmem + kT_Y + buf * 64;
+#pragma unroll
+                    for (int c0 = 0; c0 < 64; c0 += 16) {
+                        uint32_t x[16];
+                        tmem_ld16(tY + olane + c0, x);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int jj = 0; jj < 16; ++jj)
+                            sO[(c0 + jj) * kD + odv] = __float2bfloat16(p.scale * __uint_as_float(x[jj]));
+                    }
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ss.bar_yfree[buf]);     // the tile may be overwritten
+                out_sync();
+                if (ok) {
+                    const int len = min(kChunk, seq_len - j * kChunk);
+                    __nv_bfloat16* og = p.o + (static_cast<size_t>(seq_t0 + j * kChunk) * p.Hv + hv) * kD;
+#pragma unroll
+                    for (int it = 0; it < 8; ++it) {
+                        const int row = it * 8 + (ot >> 4), piece = ot & 15;
+                        if (row < len)
+                            *reinterpret_cast<uint4*>(og + row * tok_stride + piece * 8) =
+                                *reinterpret_cast<const uint4*>(sO + row * kD + piece * 8);
+                    }
+                }
+                out_sync();
+            }
         } else {
-            // ===================== epilogue warps: U and the state refresh (the dependent chain)
+            // ===================== chain warps: U and the state refresh (the dependent chain)
             // The fp32 master state lives in registers (64 per thread: row dv, columns
             // [64*half, 64*half + 64)); its bf16 copy in TMEM is the A operand of S W^T and S Qg^T.
             auto hand_over = [&](uint64_t* bar) {     // after tcgen05.st: publish to the issuing lane
@@ -456,36 +508,6 @@ __device__ __forceinline__ void fused_state_role_impl(const TensorMaps& maps, co
                     tmem_st16(tmem + kT_S + lane_base + half * 32 + (c0 >> 1), pk);
                 }
             };
-            // o rows of chunk j from Y[j & 1] in two parts that fit the two waits of the chain:
-            // (A) scale, round, transpose into shared memory; (B) whole rows in 16-byte pieces
-            auto outputs_stage = [&](int j) {
-                const uint32_t tY = tmem + kT_Y + (j & 1) * 64;
-                __nv_bfloat16* sO = reinterpret_cast<__nv_bfloat16*>(smem + kS_Out);
-#pragma unroll
-                for (int c0 = 0; c0 < 32; c0 += 16) {
-                    uint32_t x[16];
-                    tmem_ld16(tY + lane_base + half * 32 + c0, x);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int jj = 0; jj < 16; ++jj)
-                        sO[(half * 32 + c0 + jj) * kD + dv] =
-                            __float2bfloat16(p.scale * __uint_as_float(x[jj]));
-                }
-            };
-            auto outputs_flush = [&](int j) {
-                const __nv_bfloat16* sO = reinterpret_cast<const __nv_bfloat16*>(smem + kS_Out);
-                const int len = min(kChunk, seq_len - j * kChunk);
-                __nv_bfloat16* og = p.o + (static_cast<size_t>(seq_t0 + j * kChunk) * p.Hv + hv) * kD;
-                const size_t tok_stride = static_cast<size_t>(p.Hv) * kD;
-#pragma unroll
-                for (int it = 0; it < 4; ++it) {
-                    const int row = it * 16 + (tid >> 4), piece = tid & 15;
-                    if (row < len)
-                        *reinterpret_cast<uint4*>(og + row * tok_stride + piece * 8) =
-                            *reinterpret_cast<const uint4*>(sO + row * kD + piece * 8);
-                }
-            };
-
             bool ok = true;
             auto await = [&](uint64_t* bar, uint32_t parity) {   // bounded wait + tcgen05 fence
                 if (ok && !warp_wait_or_abort(bar, parity, abortp)) ok = false;
@@ -509,11 +531,6 @@ __device__ __forceinline__ void fused_state_role_impl(const TensorMaps& maps, co
             for (int j = 0; j < nc; ++j) {
                 const int st = j & 1;
                 const uint8_t* base = smem + st * kStageBytes;
-                if (j > 0) {     // part A of the previous chunk's outputs, while D1 is in flight
-                    await(&ss.bar_y, par_chunk(j - 1));
-                    epi_sync();
-                    if (ok) outputs_stage(j - 1);
-                }
                 await(&ss.bar_full[st], par_full(j));
                 await(&ss.bar_d1, par_chunk(j));
                 if (ok) {   // U^T[dv][c] = U~^T - D1 for the thread's 32 tokens [32*half, 32*half+32)
@@ -550,10 +567,6 @@ __device__ __forceinline__ void fused_state_role_impl(const TensorMaps& maps, co
                     }
                 }
                 hand_over(&ss.bar_u);
-                if (j > 0) {     // part B, while this chunk's state product is in flight
-                    epi_sync();
-                    if (ok) outputs_flush(j - 1);
-                }
                 const bool last = j + 1 == nc;
                 await(&ss.bar_d4, par_chunk(j));
                 if (ok) {   // S <- e^{b_C} S + D4 on the thread's 64 dk columns
@@ -582,11 +595,6 @@ __device__ __forceinline__ void fused_state_role_impl(const TensorMaps& maps, co
                 if (lane == 0) mbar_arrive(&ss.bar_free[st]);     // this warp is done with the stage
                 hand_over(&ss.bar_s);
             }
-            await(&ss.bar_y, par_chunk(nc - 1));
-            epi_sync();
-            if (ok) outputs_stage(nc - 1);
-            epi_sync();
-            if (ok) outputs_flush(nc - 1);
         }
         tc_fence_before_sync();
         role_sync();                                   // end of the unit: barriers are re-armed next
@@ -604,18 +612,25 @@ __device__ __forceinline__ void fused_state_role(const TensorMaps& maps, const P
                                                  uint8_t* smem, StateStatics& ss,
                                                  const uint32_t tmem) {
     // The kernel is compiled for 768 threads (80 registers each) because of the producer CTAs.
-    // In a state-pass CTA the fourteen spare warps and the issuing / loading warps hand most of
-    // their registers back and the eight chain warps take 168 each, enough to keep the fp32
-    // master state in registers (setmaxnreg works on groups of four warps).
+    // In a state-pass CTA the spare warps, the issuing / loading group and the output warps hand
+    // registers back and the eight chain warps take 160 each, enough to keep the fp32 master
+    // state in registers.  setmaxnreg works on groups of four warps and WAITS, unbounded, until
+    // the registers it asks for are free, so the budget must hold with room to spare: all counts
+    // are multiples of 16 (the allocation unit may be that coarse); 768 x 80 leaves 4096 of the
+    // 65536 registers free, the groups give back 256 x 48 + 128 x 32 + 128 x 32 = 20480 more, the
+    // chain warps take 256 x 80 = 20480.
     const int warp = threadIdx.x >> 5;
-    if (warp >= 12) {
-        reg_dealloc<24>();                            // spare warps of the CTA
+    if (warp >= 16) {
+        reg_dealloc<32>();                            // spare warps of the CTA
+    } else if (warp >= kFOutWarp0) {
+        reg_dealloc<48>();
+        fused_state_role_impl<2>(maps, p, ws, lay, smem, ss, tmem);
     } else if (warp >= 8) {
-        reg_dealloc<64>();
-        if (warp <= kFLoadWarp) fused_state_role_impl<false>(maps, p, ws, lay, smem, ss, tmem);
+        reg_dealloc<48>();
+        if (warp <= kFLoadWarp) fused_state_role_impl<0>(maps, p, ws, lay, smem, ss, tmem);
     } else {
-        reg_alloc<168>();
-        fused_state_role_impl<true>(maps, p, ws, lay, smem, ss, tmem);
+        reg_alloc<160>();
+        fused_state_role_impl<1>(maps, p, ws, lay, smem, ss, tmem);
     }
 }
 
