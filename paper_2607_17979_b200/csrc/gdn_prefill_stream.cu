@@ -13,7 +13,7 @@
 //   * warps 8-11 (output) turn Y = S Qg^T + U P^T into o rows one chunk behind, so that no
 //     output work sits in the chain warps' instruction stream (it cost about 500 of the 4300
 //     cycles of a chunk step there).
-// The CTA is compiled for 512 threads (128 registers); the chain warps take 168 registers each
+// The CTA is compiled for 512 threads (128 registers); the chain warps take 160 registers each
 // from what the other groups hand back (setmaxnreg).
 // The roles never meet at a CTA barrier inside the loop: each derives the same unit list
 // (unit = blockIdx.x + i * gridDim.x over the rank-sorted units, longest sequences first) and the
@@ -125,8 +125,11 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
     // and one after every chunk but the unit's last).
     uint32_t gc = 0;
 
+    // Register budget (setmaxnreg waits, unbounded, for what it asks: keep room to spare and use
+    // multiples of 16): 512 x 128 registers are the whole file; the issuing group gives back
+    // 128 x 80, the output warps 128 x 48, the chain warps take 256 x 32.
     if (warp >= kSIssueWarp) {
-    reg_dealloc<56>();
+    reg_dealloc<48>();
     if (warp == kSLoadWarp) {
         // ===================== loader: records and K tiles, in stream order
         if (lane == 0) {
@@ -250,7 +253,7 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
         __syncwarp();
     }
     } else if (warp < kSEpiWarps) {
-        reg_alloc<168>();
+        reg_alloc<160>();
         // ===================== chain warps: U and the state refresh (the dependent chain)
         auto hand_over = [&](uint64_t* bar) {     // after tcgen05.st: publish to the issuing lane
             tmem_wait_st();
