@@ -220,17 +220,18 @@ def test_thousands_of_tiny_sequences():
         U.check_state(S.astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
 
 
-def test_chunked_repeatable_under_load_many_ctas():
+@pytest.mark.parametrize("impl", ["chunked", "stream", "fused"])
+def test_chunked_repeatable_under_load_many_ctas(impl):
     """Several back-to-back runs of a batch that fills the GPU (64 sequence-heads, ragged tails,
     last chunks of every length class) must be bit-identical: a missed barrier between the
     kernel's warp roles shows up as run-to-run differences long before it shows up as a large
     error."""
     lens = [448, 449, 511, 512, 513, 1000, 77, 1536]
     p = I.prefill_inputs(lens, 4, 8, seed=1234, init="normal")
-    ref_o, ref_S, st = run_prefill(p, "chunked")
+    ref_o, ref_S, st = run_prefill(p, impl)
     assert st == 0
     for _ in range(4):
-        o, S, st = run_prefill(p, "chunked")
+        o, S, st = run_prefill(p, impl)
         assert st == 0 and np.array_equal(o, ref_o) and np.array_equal(S, ref_S)
     o_ref, S_ref, _ = oracle_prefill(p)
     U.check_o(ref_o, o_ref, U.O_REL_L2_PREFILL)
