@@ -88,9 +88,11 @@ __device__ __forceinline__ void mma_tile_tf32x3(const float* A, int lda, const f
 // off-diagonal blocks by block elimination at block sizes 16 and 32
 //     [[Ta, 0], [X, Tb]],  X = -Tb (A_ba Ta),
 // whose small products run on the legacy mma.sync path with split-tf32 operands (fp32-level
-// accuracy; tcgen05 needs M >= 64).  Ends with a __syncthreads().
+// accuracy; tcgen05 needs M >= 64).  Rows past the chunk's length `len` are zero in A, so the
+// elimination levels that only touch such rows are skipped.  Ends with a group barrier.
 template <class Sync>
-__device__ __forceinline__ void solve_unit_lower_64(float* sA, float* scr, int tid, Sync sync) {
+__device__ __forceinline__ void solve_unit_lower_64(float* sA, float* scr, int tid, Sync sync,
+                                                    const int len = 64) {
     // ---- diagonal blocks: thread (I, j) computes column j of (I + A_II)^{-1}, right-looking
     if (tid < 64) {
         const int I = tid >> 4, j = tid & 15;
@@ -111,6 +113,7 @@ __device__ __forceinline__ void solve_unit_lower_64(float* sA, float* scr, int t
     // the scratch borrows shared memory whose previous contents thread 0 is still bulk-storing
     if (tid == 0) bulk_wait_read_all();
     sync();
+    if (len <= 16) return;                 // every off-diagonal block lies in zero rows
     // ---- off-diagonal blocks on the tensor cores (mma.sync m16n8k8, 3xTF32: fp32-level accuracy)
     const int warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     // 16-blocks (1,0) and (3,2): X = A_IJ T_JJ, then T_IJ = -T_II X.  Four 16x8 tiles, warps 0-3.
@@ -135,6 +138,7 @@ __device__ __forceinline__ void solve_unit_lower_64(float* sA, float* scr, int t
         }
     }
     sync();
+    if (len <= 32) return;                 // block (1,0) of the 32-level lies in zero rows
     // 32-block (1,0): Y = A_ba Ta, then X = -Tb Y.  Eight 16x8 tiles, one per warp.
     {
         const int mr = warp >> 2, nb = warp & 3;
@@ -346,7 +350,7 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
         bulk_commit();
     }
 
-    solve_unit_lower_64(sA, reinterpret_cast<float*>(smem + kI_Scr), tid, sync);
+    solve_unit_lower_64(sA, reinterpret_cast<float*>(smem + kI_Scr), tid, sync, ci.len);
 
     uint32_t tu_lo[2][4];    // T diag(beta) - bf16(T diag(beta)), parked until T_w is dead
     {   // T (fp32, row-major) -> bf16 B operands T diag(beta e^b), T diag(beta) (hi, lo)
@@ -389,10 +393,12 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
         tma_load_2d(smem + kI_V + 8192, &maps.v, hv * kD + 64, ci.t0, &st.bar_v);
         const uint32_t idesc = make_idesc_bf16(128, 64, true, false);
         const uint32_t sTw = smem_u32(smem + kI_Tw);
+        // columns of T_w and T_u past the chunk's length are zero: their k-steps are left out
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks)
-            mma_ss(tW, make_sdesc_sw128(sQK + 8192 + ks * 2048, 16384, 1024),
-                   make_sdesc_sw128(sTw + ks * 32, 16, 1024), idesc, ks > 0);
+            if (ks * 16 < ci.len)
+                mma_ss(tW, make_sdesc_sw128(sQK + 8192 + ks * 2048, 16384, 1024),
+                       make_sdesc_sw128(sTw + ks * 32, 16, 1024), idesc, ks > 0);
         mma_commit(&st.bar_mma);
     }
     if (warp == 0 && !warp_wait(&st.bar_mma, par3 ^ 1u)) st.abort_flag = 1;
@@ -444,12 +450,14 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
         const uint32_t sTu = smem_u32(smem + kI_Tu), sTuLo = smem_u32(smem + kI_TuLo);
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks)
-            mma_ss(tU, make_sdesc_sw128(sV + ks * 2048, 8192, 1024),
-                   make_sdesc_sw128(sTu + ks * 32, 16, 1024), idesc, ks > 0);
+            if (ks * 16 < ci.len)
+                mma_ss(tU, make_sdesc_sw128(sV + ks * 2048, 8192, 1024),
+                       make_sdesc_sw128(sTu + ks * 32, 16, 1024), idesc, ks > 0);
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks)
-            mma_ss(tU, make_sdesc_sw128(sV + ks * 2048, 8192, 1024),
-                   make_sdesc_sw128(sTuLo + ks * 32, 16, 1024), idesc, true);
+            if (ks * 16 < ci.len)
+                mma_ss(tU, make_sdesc_sw128(sV + ks * 2048, 8192, 1024),
+                       make_sdesc_sw128(sTuLo + ks * 32, 16, 1024), idesc, true);
         mma_commit(&st.bar_mma);
     }
     if (warp == 0 && !warp_wait(&st.bar_mma, par3)) st.abort_flag = 1;
