@@ -204,9 +204,19 @@ int gdn_prefill(const void* q, const void* k, const void* v,
  * chunked variants (gdn_prefill_fused for a few long sequence-heads,
  * gdn_prefill_stream from about half a sequence-head per SM up, else
  * gdn_prefill_chunked).  Each route can also be called directly; arguments
- * are gdn_prefill's.
+ * are gdn_prefill's.  gdn_prefill_route answers which one gdn_prefill would take
+ * (host-only arithmetic on the shapes; sm_count and cooperative_launch describe
+ * the device, gdn_prefill itself queries them): one of GDN_ROUTE_*, or
+ * GDN_ROUTE_NONE for an empty batch.
  */
 #define GDN_RECURRENT_MAX_SEQLEN 16
+#define GDN_ROUTE_NONE      0
+#define GDN_ROUTE_RECURRENT 1
+#define GDN_ROUTE_CHUNKED   2
+#define GDN_ROUTE_FUSED     3
+#define GDN_ROUTE_STREAM    4
+int gdn_prefill_route(int32_t T, int32_t N, int32_t max_seqlen_hint, int32_t Hv,
+                      int32_t sm_count, int32_t cooperative_launch);
 int gdn_prefill_chunked(const void* q, const void* k, const void* v,
                         const float* g, const float* beta, const int32_t* cu_seqlens,
                         const float* init_state, float* final_state, const int32_t* slot_idx,

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libgdn_b200.so")
 
 EXPORTS = ("gdn_decode", "gdn_prefill_workspace_bytes", "gdn_prefill", "gdn_prefill_chunked",
-           "gdn_prefill_fused", "gdn_prefill_stream", "gdn_decode_multi", "gdn_gate",
+           "gdn_prefill_fused", "gdn_prefill_stream", "gdn_prefill_route", "gdn_decode_multi", "gdn_gate",
            "gdn_state_transpose", "gdn_decode_host", "gdn_decode_host_staging_bytes",
            "gdn_prefill_host", "gdn_prefill_host_staging_bytes",
            "gdn_prefill_recurrent",
@@ -51,6 +51,8 @@ _lib.gdn_prefill_chunked.restype = ctypes.c_int
 _lib.gdn_prefill_chunked.argtypes = _lib.gdn_prefill.argtypes
 _lib.gdn_prefill_fused.restype = ctypes.c_int
 _lib.gdn_prefill_fused.argtypes = _lib.gdn_prefill.argtypes
+_lib.gdn_prefill_route.restype = ctypes.c_int
+_lib.gdn_prefill_route.argtypes = [_I] * 6
 _lib.gdn_prefill_stream.restype = ctypes.c_int
 _lib.gdn_prefill_stream.argtypes = _lib.gdn_prefill.argtypes
 _lib.gdn_prefill_recurrent.restype = ctypes.c_int
@@ -160,6 +162,15 @@ def gdn_state_transpose(state_pool, slot_idx=None, n=None, dev_status=None):
         int(n), Hv, dk, dv, num_slots, _dev(dev_status, torch.int32, "dev_status", True), _stream())
     if rc != 0:
         raise GdnError(rc, "gdn_state_transpose")
+
+
+ROUTES = {0: "none", 1: "recurrent", 2: "chunked", 3: "fused", 4: "stream"}
+
+
+def gdn_prefill_route(T, N, max_seqlen_hint, Hv, sm_count=148, cooperative_launch=True) -> str:
+    """Which route gdn_prefill takes for a batch of this shape on a device with sm_count SMs."""
+    return ROUTES[int(_lib.gdn_prefill_route(T, N, int(max_seqlen_hint), Hv, sm_count,
+                                             1 if cooperative_launch else 0))]
 
 
 def gdn_prefill_workspace_bytes(T, N, Hqk, Hv, dk=128, dv=128, chunk=64) -> int:

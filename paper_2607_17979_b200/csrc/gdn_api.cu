@@ -227,17 +227,37 @@ int gdn_prefill_stream(const void* q, const void* k, const void* v, const float*
                                 workspace, workspace_bytes, dev_status, stream);
 }
 
+int gdn_prefill_route(int32_t T, int32_t N, int32_t max_seqlen_hint, int32_t Hv, int32_t sm_count,
+                      int32_t cooperative_launch) {
+    if (T <= 0 || N <= 0 || Hv <= 0 || sm_count <= 0) return GDN_ROUTE_NONE;
+    // the length is known on the host only through the caller's hint or the bound T
+    const int32_t longest = (max_seqlen_hint > 0 && max_seqlen_hint < T) ? max_seqlen_hint : T;
+    // very short sequences: the token-by-token kernel (one launch, no workspace traffic)
+    if (longest <= GDN_RECURRENT_MAX_SEQLEN) return GDN_ROUTE_RECURRENT;
+    const long long units = static_cast<long long>(N) * Hv;
+    // Few (sequence, v-head) units and long sequences: the serial state pass would occupy only a
+    // few SMs while the rest idle, so run it next to the record producers in one cooperative launch.
+    if (cooperative_launch && units <= sm_count / 3 && longest > 16 * gdn::kChunk) return GDN_ROUTE_FUSED;
+    // The persistent state pass does not pay a CTA start, a pipeline fill and a drain per unit, and
+    // its loader, issuer, chain and output warps are separate; measured equal or faster from about
+    // half a unit per SM up.  Below that the plain pass has the cheaper table-building launch.
+    if (2 * units > sm_count) return GDN_ROUTE_STREAM;
+    return GDN_ROUTE_CHUNKED;
+}
+
 int gdn_prefill(const void* q, const void* k, const void* v, const float* g, const float* beta,
                 const int32_t* cu_seqlens, const float* init_state, float* final_state,
                 const int32_t* slot_idx, void* o, int32_t T, int32_t N, int32_t max_seqlen_hint,
                 int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv, int32_t chunk,
                 int32_t num_slots, float scale, void* workspace, size_t workspace_bytes,
                 int32_t* dev_status, void* stream) {
-    // Route: a batch whose longest sequence is at most GDN_RECURRENT_MAX_SEQLEN tokens goes to the
-    // token-by-token kernel (one launch, no workspace traffic); everything else is chunked.  The
-    // length is known on the host only through the caller's hint or the bound T.
-    const int32_t longest = (max_seqlen_hint > 0 && max_seqlen_hint < T) ? max_seqlen_hint : T;
-    if (chunk == gdn::kChunk && T > 0 && N > 0 && longest <= GDN_RECURRENT_MAX_SEQLEN) {
+    int dev = 0, sms = 148, coop = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) {
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+    }
+    const int route_id = gdn_prefill_route(T, N, max_seqlen_hint, Hv, sms, coop);
+    if (chunk == gdn::kChunk && route_id == GDN_ROUTE_RECURRENT) {
         // same validation of the workspace arguments as the chunked route, so that a call does
         // not start failing when its batch grows
         if (!workspace) {
@@ -253,21 +273,9 @@ int gdn_prefill(const void* q, const void* k, const void* v, const float* g, con
                                      slot_idx, o, T, N, Hqk, Hv, dk, dv, num_slots, scale,
                                      dev_status, stream);
     }
-    // Few (sequence, v-head) units: the serial state pass would occupy only a few SMs while the
-    // rest idle, so run it next to the record producers in one cooperative launch.  Many units:
-    // the three-launch path keeps every SM on one kind of work at a time and is faster.
-    int dev = 0, sms = 148, coop = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess) {
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
-    }
-    const long long units = static_cast<long long>(N) * Hv;
-    const bool few_units = units <= sms / 3 && longest > 16 * gdn::kChunk;
-    // The persistent state pass does not pay a CTA start, a pipeline fill and a drain per unit and
-    // its loader is a warp of its own; measured equal or faster from about half a unit per SM
-    // up.  Below that the plain pass has the cheaper table-building launch.
-    const bool many_units = 2 * units > sms;
-    const PrefillRoute route = coop && few_units ? kRouteFused : many_units ? kRouteStream : kRouteChunked;
+    const PrefillRoute route = route_id == GDN_ROUTE_FUSED    ? kRouteFused
+                               : route_id == GDN_ROUTE_STREAM ? kRouteStream
+                                                              : kRouteChunked;
     return prefill_chunked_impl(route, q, k, v, g, beta, cu_seqlens, init_state,
                                 final_state, slot_idx, o, T, N, Hqk, Hv, dk, dv, chunk, num_slots,
                                 scale, workspace, workspace_bytes, dev_status, stream);

@@ -96,3 +96,25 @@ def test_prefill_validation_rejects_before_launch(lib):
     need = lib.gdn_prefill_workspace_bytes(64, 1, 1, 1, 128, 128, 64)
     assert need > 0 and call(ws_bytes=need - 1) == -5
     assert lib.gdn_prefill_workspace_bytes(64, 1, 1, 1, 64, 128, 64) == 0
+
+
+def test_prefill_routing_rules_are_pure_host_arithmetic():
+    """gdn_prefill_route needs no GPU: it answers from the shapes and the two device facts it is
+    given which variant gdn_prefill would launch."""
+    from paper_2607_17979_b200 import api
+    r = api.gdn_prefill_route
+    assert r(0, 0, 0, 32) == "none" and r(100, 0, 0, 32) == "none"
+    # longest sequence (hint, else the bound T) up to 16 tokens: token by token
+    assert r(16, 1, 0, 32) == "recurrent" and r(4000, 400, 12, 32) == "recurrent"
+    assert r(17, 1, 0, 32) != "recurrent" and r(4000, 400, 17, 8) != "recurrent"
+    # a hint larger than T is ignored
+    assert r(10, 1, 5000, 32) == "recurrent"
+    # few long units: one cooperative launch, if the device can
+    assert r(32768, 1, 0, 32) == "fused" and r(32768, 1, 0, 32, 148, False) == "chunked"
+    assert r(1025, 1, 0, 32) == "fused" and r(1024, 1, 0, 32) == "chunked"
+    assert r(32768, 1, 0, 49) == "fused" and r(32768, 1, 0, 50) == "chunked"      # 148 // 3 = 49 units
+    # from half a unit per SM up: the persistent state pass
+    assert r(7680, 4, 4096, 32) == "stream" and r(4096, 2, 2048, 32) == "chunked"   # 128 / 64 units
+    assert r(8192, 57, 144, 32) == "stream" and r(512, 3, 200, 25) == "stream" and r(512, 2, 300, 37) == "chunked"
+    # the thresholds follow the SM count given
+    assert r(4096, 2, 2048, 32, 100) == "stream"
