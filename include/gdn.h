@@ -202,8 +202,8 @@ int gdn_prefill(const void* q, const void* k, const void* v,
  * GDN_RECURRENT_MAX_SEQLEN tokens (by max_seqlen_hint if given, else by the
  * bound T) goes to the token-by-token kernel; anything longer to one of the
  * chunked variants (gdn_prefill_fused for a few long sequence-heads,
- * gdn_prefill_stream from about half a sequence-head per SM up, else
- * gdn_prefill_chunked).  Each route can also be called directly; arguments
+ * gdn_prefill_stream for chains longer than two chunks or several
+ * sequence-heads per SM, else gdn_prefill_chunked).  Each route can also be called directly; arguments
  * are gdn_prefill's.  gdn_prefill_route answers which one gdn_prefill would take
  * (host-only arithmetic on the shapes; sm_count and cooperative_launch describe
  * the device, gdn_prefill itself queries them): one of GDN_ROUTE_*, or
@@ -247,8 +247,7 @@ int gdn_prefill_fused(const void* q, const void* k, const void* v,
  * gdn_prefill_stream - the chunked algorithm in three launches whose state
  * pass is a persistent kernel: one CTA per SM walks a list of (sequence,
  * v-head) units and streams their chunks without draining its pipeline
- * between units.  It is the route gdn_prefill takes for batches with more
- * units than SMs.  Arguments, workspace and results are gdn_prefill_chunked's.
+ * between units.  Arguments, workspace and results are gdn_prefill_chunked's.
  */
 int gdn_prefill_stream(const void* q, const void* k, const void* v,
                        const float* g, const float* beta, const int32_t* cu_seqlens,

@@ -238,10 +238,12 @@ int gdn_prefill_route(int32_t T, int32_t N, int32_t max_seqlen_hint, int32_t Hv,
     // Few (sequence, v-head) units and long sequences: the serial state pass would occupy only a
     // few SMs while the rest idle, so run it next to the record producers in one cooperative launch.
     if (cooperative_launch && units <= sm_count / 3 && longest > 16 * gdn::kChunk) return GDN_ROUTE_FUSED;
-    // The persistent state pass does not pay a CTA start, a pipeline fill and a drain per unit, and
-    // its loader, issuer, chain and output warps are separate; measured equal or faster from about
-    // half a unit per SM up.  Below that the plain pass has the cheaper table-building launch.
-    if (2 * units > sm_count) return GDN_ROUTE_STREAM;
+    // The persistent state pass has the shorter chunk step (its loader, issuer, chain and output
+    // warps are separate) and does not pay a CTA start, a pipeline fill and a drain per unit:
+    // measured faster whenever a chain is longer than two chunks or there are several units per
+    // SM.  Below that the plain pass, with its cheaper table-building launch, is ahead by a
+    // microsecond.
+    if (longest > 2 * gdn::kChunk || units > 4LL * sm_count) return GDN_ROUTE_STREAM;
     return GDN_ROUTE_CHUNKED;
 }
 

@@ -110,11 +110,12 @@ def test_prefill_routing_rules_are_pure_host_arithmetic():
     # a hint larger than T is ignored
     assert r(10, 1, 5000, 32) == "recurrent"
     # few long units: one cooperative launch, if the device can
-    assert r(32768, 1, 0, 32) == "fused" and r(32768, 1, 0, 32, 148, False) == "chunked"
-    assert r(1025, 1, 0, 32) == "fused" and r(1024, 1, 0, 32) == "chunked"
-    assert r(32768, 1, 0, 49) == "fused" and r(32768, 1, 0, 50) == "chunked"      # 148 // 3 = 49 units
-    # from half a unit per SM up: the persistent state pass
-    assert r(7680, 4, 4096, 32) == "stream" and r(4096, 2, 2048, 32) == "chunked"   # 128 / 64 units
-    assert r(8192, 57, 144, 32) == "stream" and r(512, 3, 200, 25) == "stream" and r(512, 2, 300, 37) == "chunked"
+    assert r(32768, 1, 0, 32) == "fused" and r(32768, 1, 0, 32, 148, False) == "stream"
+    assert r(1025, 1, 0, 32) == "fused" and r(1024, 1, 0, 32) == "stream"
+    assert r(32768, 1, 0, 49) == "fused" and r(32768, 1, 0, 50) == "stream"       # 148 // 3 = 49 units
+    # a chain longer than two chunks, or several units per SM: the persistent state pass
+    assert r(7680, 4, 4096, 32) == "stream" and r(129, 1, 0, 32) == "stream"
+    assert r(128, 1, 0, 32) == "chunked" and r(400, 4, 100, 32) == "chunked"
+    assert r(8192, 128, 64, 32) == "stream" and r(1184, 37, 32, 16) == "chunked"    # 4096 / 592 units
     # the thresholds follow the SM count given
-    assert r(4096, 2, 2048, 32, 100) == "stream"
+    assert r(1184, 37, 32, 16, 100) == "stream"
