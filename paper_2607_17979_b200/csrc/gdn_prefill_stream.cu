@@ -127,9 +127,9 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
 
     // Register budget (setmaxnreg waits, unbounded, for what it asks: keep room to spare and use
     // multiples of 16): 512 x 128 registers are the whole file; the issuing group gives back
-    // 128 x 80, the output warps 128 x 48, the chain warps take 256 x 32.
+    // 128 x 64, the output warps 128 x 48, the chain warps take 256 x 32.
     if (warp >= kSIssueWarp) {
-    reg_dealloc<48>();
+    reg_dealloc<64>();
     if (warp == kSLoadWarp) {
         // ===================== loader: records and K tiles, in stream order
         if (lane == 0) {
