@@ -305,8 +305,8 @@ prefill_state_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
                 tmem_wait_ld();
 #pragma unroll
                 for (int jj = 0; jj < 16; ++jj) {
-                    sO[(half * 32 + jj) * kD + dv] = __float2bfloat16(p.scale * __uint_as_float(x[jj]));
-                    sO[(half * 32 + 16 + jj) * kD + dv] = __float2bfloat16(p.scale * __uint_as_float(y[jj]));
+                    sO[(half * 32 + jj) * kD + dv] = __float2bfloat16(__uint_as_float(x[jj]));
+                    sO[(half * 32 + 16 + jj) * kD + dv] = __float2bfloat16(__uint_as_float(y[jj]));
                 }
             };
             auto outputs_flush = [&](int j) {

@@ -287,7 +287,7 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
         const int r = row & 63;
         const bool is_p = row < 64;
         const float br2 = st.s_b2[r];
-        const float rowscale = is_p ? 1.f : st.s_beta[r];
+        const float rowscale = is_p ? p.scale : st.s_beta[r];      // the output scale rides on P and Qg
         const int limit = is_p ? r : r - 1;              // keep columns i <= limit
 #pragma unroll
         for (int step = 0; step < 2; ++step) {
@@ -326,14 +326,14 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
             }
         }
     }
-    {   // Q rows scaled by e^{b_r}, in place (the Gram product has consumed Q): this is the Qg image
+    {   // Q rows scaled by scale * e^{b_r}, in place (the Gram product has consumed Q): this is the Qg image
 #pragma unroll
         for (int it = 0; it < 4; ++it) {
             const int idx = tid + it * kIntraThreads;          // 1024 16-byte pieces
             const int halfq = idx >> 9, rem = idx & 511;
             const int r = rem >> 3;
             uint4* ptr = reinterpret_cast<uint4*>(smem + kI_QK + halfq * 16384 + rem * 16);
-            const float f = st.s_eb[r];
+            const float f = st.s_eb[r] * p.scale;
             uint4 w = *ptr;
             w.x = scale_bf16x2(w.x, f); w.y = scale_bf16x2(w.y, f);
             w.z = scale_bf16x2(w.z, f); w.w = scale_bf16x2(w.w, f);

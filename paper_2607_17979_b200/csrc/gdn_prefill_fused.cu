@@ -468,7 +468,7 @@ __device__ __forceinline__ void fused_state_role_impl(const TensorMaps& maps, co
                         tmem_wait_ld();
 #pragma unroll
                         for (int jj = 0; jj < 16; ++jj)
-                            sO[(c0 + jj) * kD + odv] = __float2bfloat16(p.scale * __uint_as_float(x[jj]));
+                            sO[(c0 + jj) * kD + odv] = __float2bfloat16(__uint_as_float(x[jj]));
                     }
                 }
                 tc_fence_before_sync();

@@ -127,7 +127,7 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
 
     // Register budget (setmaxnreg waits, unbounded, for what it asks: keep room to spare and use
     // multiples of 16): 512 x 128 registers are the whole file; the issuing group gives back
-    // 128 x 64, the output warps 128 x 48, the chain warps take 256 x 32.
+    // 128 x 64, the output warps 128 x 16, the chain warps take 256 x 32.
     if (warp >= kSIssueWarp) {
     reg_dealloc<64>();
     if (warp == kSLoadWarp) {
@@ -389,12 +389,11 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
             gc += nc;
         }
     } else {
-        reg_dealloc<80>();
+        reg_dealloc<112>();
         // ===================== output warps: Y = S Qg^T + U P^T (fp32, TMEM) -> o rows.  Warp 8 + q
         // reads TMEM lanes 32 q .. 32 q + 31 (dv indices), scales and rounds, transposes through
         // shared memory, and the four warps write whole rows in 16-byte pieces.
         const int q4 = warp & 3;
-        const int odv = q4 * 32 + lane;
         const uint32_t olane = static_cast<uint32_t>(q4 * 32) << 16;
         const int ot = tid - kSOutWarp0 * 32;
         const size_t tok_stride = static_cast<size_t>(p.Hv) * kD;
@@ -412,31 +411,48 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
                 // every warp runs both group barriers of every chunk, also after a failed wait
                 if (ok && !warp_wait_or_abort(&bar_y[buf], (g >> 1) & 1u, abortp)) ok = false;
                 tc_fence_after_sync();
+                // The Y tile (lanes = dv, columns = tokens) is read as accumulator fragments, rounded
+                // in pairs and stored transposed, 8 dv of one token per 16 bytes, into a [token][dv]
+                // tile of two 128B-swizzled halves of 64 dv: 2 loads, 32 conversions and 8 stores
+                // per thread instead of 64 scalar conversions and 64 two-byte stores (what these
+                // warps issue comes out of the chain warps' issue slots).
+                uint32_t pa[16], pb[16];     // packed pairs: lanes 0-15 / 16-31 of the quadrant
                 if (ok) {
                     const uint32_t tY = tmem + kT_Y + buf * 64;
+                    uint32_t y[32];
+                    tmem_ld_16x256b_x8(tY + olane, y);
+                    tmem_wait_ld();
 #pragma unroll
-                    for (int c0 = 0; c0 < 64; c0 += 16) {
-                        uint32_t x[16];
-                        tmem_ld16(tY + olane + c0, x);
-                        tmem_wait_ld();
+                    for (int i = 0; i < 16; ++i)
+                        pa[i] = pack_bf16(__uint_as_float(y[2 * i]), __uint_as_float(y[2 * i + 1]));
+                    tmem_ld_16x256b_x8(tY + olane + (16u << 16), y);
+                    tmem_wait_ld();
 #pragma unroll
-                        for (int jj = 0; jj < 16; ++jj)
-                            sO[(c0 + jj) * kD + odv] = __float2bfloat16(p.scale * __uint_as_float(x[jj]));
-                    }
+                    for (int i = 0; i < 16; ++i)
+                        pb[i] = pack_bf16(__uint_as_float(y[2 * i]), __uint_as_float(y[2 * i + 1]));
                 }
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bar_yfree[buf]);     // the tile may be overwritten
+                if (ok) {
+                    const int dv0 = q4 * 32 + 8 * (lane >> 3);         // the 8 dv this lane's address covers
+                    const uint32_t dst = smem_u32(sO) + (dv0 >> 6) * 8192;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        stmatrix_x4_trans(dst + sw128_offset(8 * i + (lane & 7), (dv0 & 63) >> 3),
+                                          pa[2 * i], pa[2 * i + 1], pb[2 * i], pb[2 * i + 1]);
+                }
                 out_sync();
                 if (ok) {
                     const int len = min(kChunk, u.seq_len - j * kChunk);
                     __nv_bfloat16* og = p.o + (static_cast<size_t>(u.seq_t0 + j * kChunk) * p.Hv + u.hv) * kD;
+                    const uint8_t* src = reinterpret_cast<const uint8_t*>(sO) + ((ot & 15) >> 3) * 8192;
 #pragma unroll
                     for (int it = 0; it < 8; ++it) {
                         const int row = it * 8 + (ot >> 4), piece = ot & 15;
                         if (row < len)
                             *reinterpret_cast<uint4*>(og + row * tok_stride + piece * 8) =
-                                *reinterpret_cast<const uint4*>(sO + row * kD + piece * 8);
+                                *reinterpret_cast<const uint4*>(src + sw128_offset(row, piece & 7));
                     }
                 }
                 out_sync();
