@@ -448,7 +448,6 @@ __device__ __forceinline__ void fused_state_role_impl(const TensorMaps& maps, co
             // ===================== output warps: Y = S Qg^T + U P^T (fp32, TMEM) -> o rows, one warp
             // per TMEM lane quadrant; transposed through shared memory, written as whole rows
             const int q4 = warp & 3;
-            const int odv = q4 * 32 + lane;
             const uint32_t olane = static_cast<uint32_t>(q4 * 32) << 16;
             const int ot = tid - kFOutWarp0 * 32;
             const size_t tok_stride = static_cast<size_t>(p.Hv) * kD;
@@ -459,16 +458,25 @@ __device__ __forceinline__ void fused_state_role_impl(const TensorMaps& maps, co
                 // every warp runs both group barriers of every chunk, also after a failed wait
                 if (ok && !warp_wait_or_abort(&ss.bar_y[buf], par_full(j), abortp)) ok = false;
                 tc_fence_after_sync();
+                // The Y tile (lanes = dv, columns = tokens) is read as accumulator fragments, 16 lanes
+                // at a time, rounded in pairs and stored transposed, 8 dv of one token per 16 bytes,
+                // into a [token][dv] tile of two 128B-swizzled halves of 64 dv: far fewer
+                // instructions than scalar conversions and two-byte stores, and what these warps
+                // issue comes out of the chain warps' issue slots.
                 if (ok) {
                     const uint32_t tY = tmem + kT_Y + buf * 64;
 #pragma unroll
-                    for (int c0 = 0; c0 < 64; c0 += 16) {
-                        uint32_t x[16];
-                        tmem_ld16(tY + olane + c0, x);
+                    for (int h = 0; h < 2; ++h) {
+                        uint32_t y[32];
+                        tmem_ld_16x256b_x8(tY + olane + (static_cast<uint32_t>(16 * h) << 16), y);
                         tmem_wait_ld();
+                        const int dv0 = q4 * 32 + 16 * h + 8 * ((lane >> 3) & 1);    // 8 dv behind this lane's address
+                        const uint32_t dst = smem_u32(sO) + (dv0 >> 6) * 8192;
 #pragma unroll
-                        for (int jj = 0; jj < 16; ++jj)
-                            sO[(c0 + jj) * kD + odv] = __float2bfloat16(__uint_as_float(x[jj]));
+                        for (int i = 0; i < 8; ++i)
+                            stmatrix_x2_trans(dst + sw128_offset(8 * i + (lane & 7), (dv0 & 63) >> 3),
+                                              pack_bf16(__uint_as_float(y[4 * i]), __uint_as_float(y[4 * i + 1])),
+                                              pack_bf16(__uint_as_float(y[4 * i + 2]), __uint_as_float(y[4 * i + 3])));
                     }
                 }
                 tc_fence_before_sync();
@@ -478,12 +486,13 @@ __device__ __forceinline__ void fused_state_role_impl(const TensorMaps& maps, co
                 if (ok) {
                     const int len = min(kChunk, seq_len - j * kChunk);
                     __nv_bfloat16* og = p.o + (static_cast<size_t>(seq_t0 + j * kChunk) * p.Hv + hv) * kD;
+                    const uint8_t* src = reinterpret_cast<const uint8_t*>(sO) + ((ot & 15) >> 3) * 8192;
 #pragma unroll
                     for (int it = 0; it < 8; ++it) {
                         const int row = it * 8 + (ot >> 4), piece = ot & 15;
                         if (row < len)
                             *reinterpret_cast<uint4*>(og + row * tok_stride + piece * 8) =
-                                *reinterpret_cast<const uint4*>(sO + row * kD + piece * 8);
+                                *reinterpret_cast<const uint4*>(src + sw128_offset(row, piece & 7));
                     }
                 }
                 out_sync();
@@ -613,23 +622,24 @@ __device__ __forceinline__ void fused_state_role(const TensorMaps& maps, const P
                                                  const uint32_t tmem) {
     // The kernel is compiled for 768 threads (80 registers each) because of the producer CTAs.
     // In a state-pass CTA the spare warps, the issuing / loading group and the output warps hand
-    // registers back and the eight chain warps take 160 each, enough to keep the fp32 master
+    // registers back and the eight chain warps take 144 each, enough to keep the fp32 master
     // state in registers.  setmaxnreg works on groups of four warps and WAITS, unbounded, until
-    // the registers it asks for are free, so the budget must hold with room to spare: all counts
-    // are multiples of 16 (the allocation unit may be that coarse); 768 x 80 leaves 4096 of the
-    // 65536 registers free, the groups give back 256 x 48 + 128 x 32 + 128 x 32 = 20480 more, the
-    // chain warps take 256 x 80 = 20480.
+    // the registers it asks for have been given back by other warps of the SAME CTA (registers the
+    // SM never gave this CTA do not count: asking for more than was handed back hangs the CTA).
+    // All counts are multiples of 16 (the allocation unit may be that coarse).  Given back:
+    // 256 x 48 (spare warps) + 128 x 32 (issuing / loading) + 128 x 16 (output) = 18432; taken by
+    // the chain warps: 256 x 64 = 16384.
     const int warp = threadIdx.x >> 5;
     if (warp >= 16) {
         reg_dealloc<32>();                            // spare warps of the CTA
     } else if (warp >= kFOutWarp0) {
-        reg_dealloc<48>();
+        reg_dealloc<64>();
         fused_state_role_impl<2>(maps, p, ws, lay, smem, ss, tmem);
     } else if (warp >= 8) {
         reg_dealloc<48>();
         if (warp <= kFLoadWarp) fused_state_role_impl<0>(maps, p, ws, lay, smem, ss, tmem);
     } else {
-        reg_alloc<160>();
+        reg_alloc<144>();
         fused_state_role_impl<1>(maps, p, ws, lay, smem, ss, tmem);
     }
 }

@@ -252,6 +252,12 @@ __device__ __forceinline__ void stmatrix_x4_trans(uint32_t saddr, uint32_t m0, u
                  "r"(m0), "r"(m1), "r"(m2), "r"(m3)
                  : "memory");
 }
+// Two matrices; lanes 0-15 supply the addresses.
+__device__ __forceinline__ void stmatrix_x2_trans(uint32_t saddr, uint32_t m0, uint32_t m1) {
+    asm volatile("stmatrix.sync.aligned.m8n8.x2.trans.shared.b16 [%0], {%1, %2};" ::"r"(saddr), "r"(m0),
+                 "r"(m1)
+                 : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
