@@ -13,7 +13,7 @@
 //   * warps 8-11 (output) turn Y = S Qg^T + U P^T into o rows one chunk behind, so that no
 //     output work sits in the chain warps' instruction stream (it cost about 500 of the 4300
 //     cycles of a chunk step there).
-// The CTA is compiled for 512 threads (128 registers); the chain warps take 160 registers each
+// The CTA is compiled for 512 threads (128 registers); the chain warps take 144 registers each
 // from what the other groups hand back (setmaxnreg).
 // The roles never meet at a CTA barrier inside the loop: each derives the same unit list
 // (unit = blockIdx.x + i * gridDim.x over the rank-sorted units, longest sequences first) and the
@@ -75,7 +75,7 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                                ~static_cast<uintptr_t>(1023));
-    __shared__ uint64_t bar_full[2], bar_free_a[2], bar_free_b[2], bar_free_c[2], bar_yfree[2], bar_y[2],
+    __shared__ uint64_t bar_full[2], bar_free_a[2], bar_free_b[2], bar_free_c[2], bar_y[2],
         bar_d1, bar_d4, bar_s, bar_u;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_flag;
@@ -97,13 +97,17 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
             mbar_init(&bar_free_a[st], 1);
             mbar_init(&bar_free_b[st], kSEpiWarps);
             mbar_init(&bar_free_c[st], 1);
-            mbar_init(&bar_yfree[st], kSOutThreads / 32);   // the output warps have read the tile
         }
         mbar_init(&bar_d1, 1);
         mbar_init(&bar_d4, 1);
         mbar_init(&bar_y[0], 1);      // one per Y tile: with a single barrier the output warps could
         mbar_init(&bar_y[1], 1);      // find it two phases ahead, which a parity wait cannot tell
-        mbar_init(&bar_s, kSEpiWarps);
+        // bar_s: everything the chunk's first product needs is in TMEM: the bf16 state (one arrival
+        // per chain warp) and U~ in the accumulator (one per output warp).  The output warps copy
+        // U~ only after they have seen the record land and have read the Y tile of two chunks
+        // ago, so this one wait also tells the issuing warp that the record is in shared memory
+        // and that the Y tile may be overwritten.
+        mbar_init(&bar_s, kSEpiWarps + kSOutThreads / 32);
         mbar_init(&bar_u, kSEpiWarps);
         abort_flag = 0;
         fence_barrier_init();
@@ -125,11 +129,12 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
     // and one after every chunk but the unit's last).
     uint32_t gc = 0;
 
-    // Register budget (setmaxnreg waits, unbounded, for what it asks: keep room to spare and use
-    // multiples of 16): 512 x 128 registers are the whole file; the issuing group gives back
-    // 128 x 64, the output warps 128 x 16, the chain warps take 256 x 32.
+    // Register budget: setmaxnreg waits, unbounded, until the registers it asks for have been given
+    // back by other warps of the same CTA, so keep room to spare and use multiples of 16.  512 x 128
+    // registers are the whole file; the issuing group gives back 128 x 48, the output warps keep
+    // theirs (the call only tells the compiler their budget), the chain warps take 256 x 16.
     if (warp >= kSIssueWarp) {
-    reg_dealloc<64>();
+    reg_dealloc<80>();
     if (warp == kSLoadWarp) {
         // ===================== loader: records and K tiles, in stream order
         if (lane == 0) {
@@ -170,7 +175,7 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
         {   // the whole warp runs this warp-uniform code; one elected lane executes each tcgen05 instruction
             const uint32_t id64 = make_idesc_bf16(128, 64, false, false);
             const uint32_t id128mn = make_idesc_bf16(128, 128, false, true);
-            const uint32_t id64mn = make_idesc_bf16(128, 64, false, true);
+            const uint32_t id64mn = make_idesc_bf16(128, 64, false, true) | kIdescNegateB;
             const uint32_t sRec0 = smem_u32(smem + kS_Rec), sRec1 = sRec0 + kStageBytes;
             const uint64_t dW0 = make_sdesc_sw128(sRec0 + kRecW, 8192, 1024);
             const uint64_t dQ0 = make_sdesc_sw128(sRec0 + kRecQg, 16, 1024);
@@ -194,14 +199,14 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
                     const uint64_t w = st ? dW1 : dW0, qg = st ? dQ1 : dQ0, pp = st ? dP1 : dP0,
                                    kk = st ? dK1 : dK0;
                     const uint32_t tY = tmem + kT_Y + st * 64;
-                    if (!wait_or_abort(&bar_full[st], (g >> 1) & 1u, abortp) ||
-                        !wait_or_abort(&bar_s, g & 1u, abortp)) {      // bf16 S of this chunk in TMEM
+                    if (!wait_or_abort(&bar_s, g & 1u, abortp)) {      // record landed, bf16 S and U~ in TMEM
                         live = false;
                         break;
                     }
                     tc_fence_after_sync();
-                    // D1 = S W^T  (on the chain); W is MN-major: k-step ks reads 16 dk rows = 2048 bytes
-                    if (elect_one()) mma_ts_c<false>(tD1, tS, w, id64mn);
+                    // U = U~ - S W^T  (on the chain): the accumulator holds U~, the B operand is negated;
+                    // W is MN-major: k-step ks reads 16 dk rows = 2048 bytes
+                    if (elect_one()) mma_ts_c<true>(tD1, tS, w, id64mn);
                     if (elect_one()) mma_ts_c<true>(tD1, tS + 8, sdesc_advance(w, 2048), id64mn);
                     if (elect_one()) mma_ts_c<true>(tD1, tS + 16, sdesc_advance(w, 4096), id64mn);
                     if (elect_one()) mma_ts_c<true>(tD1, tS + 24, sdesc_advance(w, 6144), id64mn);
@@ -211,10 +216,6 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
                     if (elect_one()) mma_ts_c<true>(tD1, tS + 56, sdesc_advance(w, 14336), id64mn);
                     if (elect_one()) mma_commit(&bar_d1);
                     // Y = S Qg^T  (off the chain) overwrites the tile the output warps read two chunks ago
-                    if (g >= 2 && !wait_or_abort(&bar_yfree[st], ((g - 2) >> 1) & 1u, abortp)) {
-                        live = false;
-                        break;
-                    }
                     if (elect_one()) mma_ts_c<false>(tY, tS, qg, id64);
                     if (elect_one()) mma_ts_c<true>(tY, tS + 8, sdesc_advance(qg, 32), id64);
                     if (elect_one()) mma_ts_c<true>(tY, tS + 16, sdesc_advance(qg, 64), id64);
@@ -253,7 +254,7 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
         __syncwarp();
     }
     } else if (warp < kSEpiWarps) {
-        reg_alloc<160>();
+        reg_alloc<144>();
         // ===================== chain warps: U and the state refresh (the dependent chain)
         auto hand_over = [&](uint64_t* bar) {     // after tcgen05.st: publish to the issuing lane
             tmem_wait_st();
@@ -324,8 +325,7 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
                 const uint8_t* base = smem + st * kStageBytes;
                 await(&bar_full[st], (g >> 1) & 1u);
                 await(&bar_d1, g & 1u);
-                if (ok) {   // U^T[dv][c] = U~^T - D1 for the thread's 32 tokens [32*half, 32*half+32)
-                    const float4* sU = reinterpret_cast<const float4*>(base + kS_Rec + kRecU);
+                if (ok) {   // U^T[dv][c] (the accumulator holds U~ - S W^T) for the thread's 32 tokens [32*half, 32*half+32)
                     const float* sdec = reinterpret_cast<const float*>(base + kS_Rec + kRecDecay);
 #pragma unroll
                     for (int c0 = 0; c0 < 32; c0 += 16) {
@@ -336,12 +336,11 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
                         uint32_t pu[8], ph[8], pl[8];
 #pragma unroll
                         for (int q4 = 0; q4 < 4; ++q4) {
-                            const float4 ut = sU[((cb >> 2) + q4) * kD + dv];
                             const float4 dd = *reinterpret_cast<const float4*>(sdec + cb + 4 * q4);
-                            const float u0 = ut.x - __uint_as_float(x[4 * q4 + 0]);
-                            const float u1 = ut.y - __uint_as_float(x[4 * q4 + 1]);
-                            const float u2 = ut.z - __uint_as_float(x[4 * q4 + 2]);
-                            const float u3 = ut.w - __uint_as_float(x[4 * q4 + 3]);
+                            const float u0 = __uint_as_float(x[4 * q4 + 0]);
+                            const float u1 = __uint_as_float(x[4 * q4 + 1]);
+                            const float u2 = __uint_as_float(x[4 * q4 + 2]);
+                            const float u3 = __uint_as_float(x[4 * q4 + 3]);
                             const float s0 = u0 * dd.x, s1 = u1 * dd.y, s2 = u2 * dd.z, s3 = u3 * dd.w;
                             pu[2 * q4] = pack_bf16(u0, u1);
                             pu[2 * q4 + 1] = pack_bf16(u2, u3);
@@ -389,7 +388,7 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
             gc += nc;
         }
     } else {
-        reg_dealloc<112>();
+        reg_dealloc<128>();
         // ===================== output warps: Y = S Qg^T + U P^T (fp32, TMEM) -> o rows.  Warp 8 + q
         // reads TMEM lanes 32 q .. 32 q + 31 (dv indices), scales and rounds, transposes through
         // shared memory, and the four warps write whole rows in 16-byte pieces.
@@ -400,6 +399,34 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
         __nv_bfloat16* sO = reinterpret_cast<__nv_bfloat16*>(smem + kS_Out);
         auto out_sync = [] { asm volatile("bar.sync 1, %0;" ::"n"(kSOutThreads) : "memory"); };
         bool ok = true;
+        // U~ (fp32, 32 KB per chunk) reaches the chain through the accumulator of S W^T: this group
+        // copies it from the record into TMEM one chunk ahead, the product then subtracts S W^T
+        // from it (negated B operand), and the chain warps read U itself.  (Read by the chain warps
+        // from shared memory, the 32 KB took 300 of the 3700 cycles of a chunk step.)
+        const int odv = q4 * 32 + lane;
+        auto preload = [&](uint32_t gq) {       // chunk gq of the CTA's stream -> accumulator
+            const int sq = gq & 1;
+            if (ok && !warp_wait_or_abort(&bar_full[sq], (gq >> 1) & 1u, abortp)) ok = false;
+            if (ok) {
+                const float4* sU = reinterpret_cast<const float4*>(smem + sq * kStageBytes + kS_Rec + kRecU);
+#pragma unroll
+                for (int c0 = 0; c0 < 64; c0 += 16) {
+                    uint32_t r[16];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float4 v = sU[((c0 >> 2) + q) * kD + odv];
+                        r[4 * q] = __float_as_uint(v.x); r[4 * q + 1] = __float_as_uint(v.y);
+                        r[4 * q + 2] = __float_as_uint(v.z); r[4 * q + 3] = __float_as_uint(v.w);
+                    }
+                    tmem_st16(tmem + kT_D1 + olane + c0, r);
+                }
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar_s);
+        };
+        bool preloaded = false;     // U~ of the chunk about to be processed is already in place
         UnitInfo nxt = unit_info(p, ws, lay, min(static_cast<int>(blockIdx.x), total_units - 1));
         for (int unit = blockIdx.x; unit < total_units; unit += gridDim.x) {
             const UnitInfo u = nxt;
@@ -408,6 +435,21 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
             for (int j = 0; j < u.nc; ++j) {
                 const uint32_t g = gc + j;
                 const int buf = g & 1;
+                // k = 0: this chunk's U~ (first chunk of the stream, or after a skipped unit).
+                // k = 1: once the chain warps have read U of this chunk the accumulator is free for
+                // the next chunk's U~ (when the next chunk is known without looking past a skipped
+                // unit), which is then in place long before the chain warps hand the state over.
+                const bool ahead = j + 1 < u.nc || (unit + static_cast<int>(gridDim.x) < total_units && !nxt.skip);
+#pragma unroll 1
+                for (int k = preloaded ? 1 : 0; k < 2; ++k) {
+                    if (k == 1) {
+                        if (ok && !warp_wait_or_abort(&bar_u, g & 1u, abortp)) ok = false;
+                        tc_fence_after_sync();
+                        if (!ahead) break;
+                    }
+                    preload(g + k);
+                }
+                preloaded = ahead;
                 // every warp runs both group barriers of every chunk, also after a failed wait
                 if (ok && !warp_wait_or_abort(&bar_y[buf], (g >> 1) & 1u, abortp)) ok = false;
                 tc_fence_after_sync();
@@ -431,9 +473,6 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
                     for (int i = 0; i < 16; ++i)
                         pb[i] = pack_bf16(__uint_as_float(y[2 * i]), __uint_as_float(y[2 * i + 1]));
                 }
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&bar_yfree[buf]);     // the tile may be overwritten
                 if (ok) {
                     const int dv0 = q4 * 32 + 8 * (lane >> 3);         // the 8 dv this lane's address covers
                     const uint32_t dst = smem_u32(sO) + (dv0 >> 6) * 8192;

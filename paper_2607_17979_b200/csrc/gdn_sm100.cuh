@@ -138,6 +138,9 @@ __device__ __forceinline__ uint64_t make_sdesc_sw128(uint32_t smem_addr, uint32_
            (static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
 }
 
+// Bit 14 of the instruction descriptor negates the B operand: D (+)= A (-B).
+constexpr uint32_t kIdescNegateB = 1u << 14;
+
 // ------------------------------------------------------------------ MMA
 // D[tmem] (+)= A[smem] * B[smem]; issue from ONE thread.
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
