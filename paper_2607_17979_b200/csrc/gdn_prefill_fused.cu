@@ -621,25 +621,25 @@ __device__ __forceinline__ void fused_state_role(const TensorMaps& maps, const P
                                                  uint8_t* smem, StateStatics& ss,
                                                  const uint32_t tmem) {
     // The kernel is compiled for 768 threads (80 registers each) because of the producer CTAs.
-    // In a state-pass CTA the spare warps, the issuing / loading group and the output warps hand
-    // registers back and the eight chain warps take 144 each, enough to keep the fp32 master
-    // state in registers.  setmaxnreg works on groups of four warps and WAITS, unbounded, until
-    // the registers it asks for have been given back by other warps of the SAME CTA (registers the
-    // SM never gave this CTA do not count: asking for more than was handed back hangs the CTA).
-    // All counts are multiples of 16 (the allocation unit may be that coarse).  Given back:
-    // 256 x 48 (spare warps) + 128 x 32 (issuing / loading) + 128 x 16 (output) = 18432; taken by
-    // the chain warps: 256 x 64 = 16384.
+    // In a state-pass CTA the spare warps and the issuing / loading group hand registers back and
+    // the eight chain warps take 128 each, enough to keep the fp32 master state in registers.
+    // setmaxnreg works on groups of four warps and WAITS, unbounded, until the registers it asks
+    // for have been given back by other warps of the SAME CTA (registers the SM never gave this CTA
+    // do not count: asking for more than was handed back hangs the CTA).  All counts are multiples
+    // of 16 (the allocation unit may be that coarse).  Given back: 256 x 48 (spare warps) +
+    // 128 x 16 (issuing / loading) = 14336, the output warps keep their 80 (the call only tells
+    // the compiler their budget); taken by the chain warps: 256 x 48 = 12288.
     const int warp = threadIdx.x >> 5;
     if (warp >= 16) {
         reg_dealloc<32>();                            // spare warps of the CTA
     } else if (warp >= kFOutWarp0) {
-        reg_dealloc<64>();
+        reg_dealloc<80>();
         fused_state_role_impl<2>(maps, p, ws, lay, smem, ss, tmem);
     } else if (warp >= 8) {
-        reg_dealloc<48>();
+        reg_dealloc<64>();
         if (warp <= kFLoadWarp) fused_state_role_impl<0>(maps, p, ws, lay, smem, ss, tmem);
     } else {
-        reg_alloc<144>();
+        reg_alloc<128>();
         fused_state_role_impl<1>(maps, p, ws, lay, smem, ss, tmem);
     }
 }
