@@ -38,7 +38,7 @@ TILE_BYTES = 128 * 128 * 4
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures
 # (profiles/); None until a capture of that kernel exists.
-NCU_TRAFFIC_BYTES = {"decode": 213_381_376, "prefill": 730_005_760}
+NCU_TRAFFIC_BYTES = {"decode": 213_381_376, "prefill": 730_488_832}
 
 
 def peaks():
