@@ -176,7 +176,10 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
                             __nanosleep(64);
                         }
                         if (v != 1) { *abortp = 1; live = false; break; }
-                        fence_proxy_async_all();
+                        // No proxy fence here: the producer put one between its generic stores and
+                        // the flag's release, which is on the path from those stores to the copies
+                        // below; one here would also wait for this thread's copies in flight (3 %
+                        // of a long sequence's run time).
                     }
                     if (g >= 2 && !wait_or_abort(&bar_free_a[st], par_free, abortp)) { live = false; break; }
                     mbar_expect_tx(&bar_full[st], kRecBytes + 16384);
