@@ -1,28 +1,33 @@
-// Inter-chunk state pass as a PERSISTENT kernel: one CTA per SM walks a fixed list of
+// Inter-chunk state pass as a PERSISTENT role: a CTA of 512 threads walks a fixed list of
 // (sequence, v-head) units and streams their chunk records through one two-stage pipeline that
-// does not drain between units.
+// does not drain between units.  Two kernels run it: the persistent state pass after the
+// intra-chunk kernel (one CTA per SM), and the state CTAs of the fused cooperative launch, whose
+// records are produced by other CTAs while the pass runs.
 //
 // The one-CTA-per-unit state kernel pays, for every unit, a launch slot, barrier and TMEM set-up,
 // the first record's memory latency and the tail of its last chunk; with thousands of short
 // units (many short sequences) that overhead is longer than the chunk steps themselves.  Here
 //   * warp 13 (loader) copies records and K tiles in unit order, running up to two chunks ahead
-//     of the consumers and straight across unit boundaries;
+//     of the consumers and straight across unit boundaries (in the fused launch it first waits
+//     for each record's flag);
 //   * warp 12 (issuer) issues every tcgen05.mma;
-//   * warps 0-7 (chain) carry the dependent chain  D1 = S W^T -> U = U~ - D1 ->
-//     D4 = (U decayed)^T K -> S = e^{b_C} S + D4 and nothing else;
-//   * warps 8-11 (output) turn Y = S Qg^T + U P^T into o rows one chunk behind, so that no
-//     output work sits in the chain warps' instruction stream (it cost about 500 of the 4300
-//     cycles of a chunk step there).
+//   * warps 0-7 (chain) carry the dependent chain  U = U~ - S W^T  ->  D4 = (U decayed)^T K  ->
+//     S = e^{b_C} S + D4  and nothing else; U~ is already in the accumulator of S W^T when the
+//     product runs (negated B operand), so the chain warps read U itself;
+//   * warps 8-11 (output) put U~ of the next chunk into that accumulator and turn
+//     Y = S Qg^T + U P^T into o rows one chunk behind.  Whatever these warps issue comes out of
+//     the chain warps' issue slots, so the rows are made with few instructions (fragment loads,
+//     paired conversions, transposing matrix stores).
 // The CTA is compiled for 512 threads (128 registers); the chain warps take 144 registers each
 // from what the other groups hand back (setmaxnreg).
 // The roles never meet at a CTA barrier inside the loop: each derives the same unit list
-// (unit = blockIdx.x + i * gridDim.x over the rank-sorted units, longest sequences first) and the
-// same running chunk count, from which every mbarrier parity follows.  Every barrier phase is
-// consumed by its waiter before the next one can complete (a parity wait cannot tell a barrier
-// that is two phases ahead), which is why the state hand-over after a unit's last chunk is
-// omitted rather than left unconsumed.
+// (unit = cta + i * n_ctas over the rank-sorted units, longest sequences first) and the same
+// running chunk count, from which every mbarrier parity follows.  Every barrier phase is consumed
+// by its waiters before the next one can complete (a parity wait cannot tell a barrier that is two
+// phases ahead), which is why the state hand-over after a unit's last chunk is omitted rather than
+// left unconsumed.
 //
-// The fp32 master state lives in the epilogue threads' registers (64 per thread; TMEM lane = state
+// The fp32 master state lives in the chain threads' registers (64 per thread; TMEM lane = state
 // row, two column halves), as in the one-CTA-per-unit state kernel.
 #pragma once
 #include "gdn_prefill_device.cuh"
