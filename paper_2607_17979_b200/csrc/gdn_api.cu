@@ -240,10 +240,10 @@ int gdn_prefill_route(int32_t T, int32_t N, int32_t max_seqlen_hint, int32_t Hv,
     if (cooperative_launch && units <= sm_count / 3 && longest > 16 * gdn::kChunk) return GDN_ROUTE_FUSED;
     // The persistent state pass has the shorter chunk step (its loader, issuer, chain and output
     // warps are separate) and does not pay a CTA start, a pipeline fill and a drain per unit:
-    // measured faster whenever a chain is longer than two chunks or there are several units per
-    // SM.  Below that the plain pass, with its cheaper table-building launch, is ahead by a
-    // microsecond.
-    if (longest > 2 * gdn::kChunk || units > 4LL * sm_count) return GDN_ROUTE_STREAM;
+    // measured faster whenever a chain is longer than two chunks or there are more units than
+    // SMs.  Below that the plain pass, with its cheaper table-building launch, is ahead by a
+    // microsecond or two.
+    if (longest > 2 * gdn::kChunk || units > sm_count) return GDN_ROUTE_STREAM;
     return GDN_ROUTE_CHUNKED;
 }
 
