@@ -211,6 +211,10 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
         tma_load_2d(smem + kI_QK + 8192, &maps.k, hqk * kD, ci.t0, &st.bar_tma);
         tma_load_2d(smem + kI_QK + 16384, &maps.q, hqk * kD + 64, ci.t0, &st.bar_tma);
         tma_load_2d(smem + kI_QK + 24576, &maps.k, hqk * kD + 64, ci.t0, &st.bar_tma);
+        // V has no room in shared memory until the solve is over; fetch it into L2 meanwhile, so
+        // that its load then is not a DRAM round trip in front of the U~ product
+        tma_prefetch_2d(&maps.v, hv * kD, ci.t0);
+        tma_prefetch_2d(&maps.v, hv * kD + 64, ci.t0);
     }
     if (warp == 1) {
         // inclusive prefix sum of the log gates over the chunk (two tokens per lane); rows past
