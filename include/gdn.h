@@ -202,8 +202,8 @@ int gdn_prefill(const void* q, const void* k, const void* v,
  * GDN_RECURRENT_MAX_SEQLEN tokens (by max_seqlen_hint if given, else by the
  * bound T) goes to the token-by-token kernel; anything longer to one of the
  * chunked variants (gdn_prefill_fused for a few long sequence-heads,
- * gdn_prefill_stream for chains longer than two chunks or more
- * sequence-heads than SMs, else gdn_prefill_chunked).  Each route can also be called directly; arguments
+ * gdn_prefill_stream for chains longer than two chunks, more
+ * sequence-heads than SMs or at most 16 sequences, else gdn_prefill_chunked).  Each route can also be called directly; arguments
  * are gdn_prefill's.  gdn_prefill_route answers which one gdn_prefill would take
  * (host-only arithmetic on the shapes; sm_count and cooperative_launch describe
  * the device, gdn_prefill itself queries them): one of GDN_ROUTE_*, or

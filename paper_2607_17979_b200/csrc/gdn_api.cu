@@ -241,9 +241,10 @@ int gdn_prefill_route(int32_t T, int32_t N, int32_t max_seqlen_hint, int32_t Hv,
     // The persistent state pass has the shorter chunk step (its loader, issuer, chain and output
     // warps are separate) and does not pay a CTA start, a pipeline fill and a drain per unit:
     // measured faster whenever a chain is longer than two chunks or there are more units than
-    // SMs.  Below that the plain pass, with its cheaper table-building launch, is ahead by a
-    // microsecond or two.
-    if (longest > 2 * gdn::kChunk || units > sm_count) return GDN_ROUTE_STREAM;
+    // SMs, and for every batch of few sequences (no table-building launch then).  What is left,
+    // many short sequences of few heads, goes to the plain pass with its cheaper table-building
+    // launch, ahead there by a microsecond or two.
+    if (longest > 2 * gdn::kChunk || units > sm_count || N <= gdn::kInlineTableSeqs) return GDN_ROUTE_STREAM;
     return GDN_ROUTE_CHUNKED;
 }
 

@@ -40,6 +40,11 @@ constexpr uint32_t kRecDecay = 73728;
 constexpr uint32_t kRecGammaC = 73984;
 constexpr uint32_t kRecBytes = 74240;
 
+// Small batches of at most this many sequences need no table-building launch: the intra-chunk
+// kernel finds its chunks from cu_seqlens itself and writes the per-sequence tables for the state pass.
+constexpr int kInlineTableSeqs = 16;
+constexpr int kInlineTableItems = 2 * 148 * 4;     // and at most about two waves of (chunk, v-head) CTAs
+
 struct ChunkInfo {      // 16 bytes
     int32_t seq;        // sequence the chunk belongs to
     int32_t t0;         // first packed token of the chunk

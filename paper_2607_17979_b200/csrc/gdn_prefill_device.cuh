@@ -36,7 +36,12 @@ struct TensorMaps {
 // Host side: 2-D maps over the packed q, k, v (64 x 64 boxes, 128B swizzle); false on failure.
 bool make_prefill_tensor_maps(TensorMaps* maps, const PrefillParams& p);
 // Launch of the intra-chunk kernel over every (chunk, v-head) item of the batch.
-cudaError_t launch_prefill_intra(const TensorMaps& maps, const ChunkedParams& cp, cudaStream_t stream);
+// inline_tables: no table-building launch went before; every CTA finds its chunk from cu_seqlens and
+// one CTA writes the per-sequence tables (first chunk, validity, rank) for the state pass.  Only
+// for batches of few sequences: see prefill_tables_inline().
+cudaError_t launch_prefill_intra(const TensorMaps& maps, const ChunkedParams& cp, cudaStream_t stream,
+                                 bool inline_tables);
+bool prefill_tables_inline(const ChunkedParams& cp);
 
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;

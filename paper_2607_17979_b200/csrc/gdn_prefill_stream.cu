@@ -38,10 +38,13 @@ cudaError_t launch_prefill_stream(const ChunkedParams& cp, cudaStream_t stream) 
     if (e != cudaSuccess) return e;
     TensorMaps maps;
     if (!make_prefill_tensor_maps(&maps, p)) return cudaErrorInvalidValue;
-    e = launch_prefill_ranked_prep(cp, stream, false);
-    if (e != cudaSuccess) return e;
+    const bool inline_tables = prefill_tables_inline(cp);
+    if (!inline_tables) {
+        e = launch_prefill_ranked_prep(cp, stream, false);
+        if (e != cudaSuccess) return e;
+    }
     if (cp.lay.max_chunks > 0) {
-        e = launch_prefill_intra(maps, cp, stream);
+        e = launch_prefill_intra(maps, cp, stream, inline_tables);
         if (e != cudaSuccess) return e;
     }
     const long long units = static_cast<long long>(p.N) * p.Hv;
