@@ -272,3 +272,29 @@ def test_length_routed_entry_point_small_shapes(lens):
     p = I.prefill_inputs(lens, 2, 4, seed=5000 + sum(lens), init="normal")
     o, S, o_ref, S_ref = compare(p, "auto")
     U.check_state(S.astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
+
+
+@pytest.mark.parametrize("impl", ["auto", "chunked", "stream"])
+@pytest.mark.parametrize("N", [16, 17])
+def test_small_batches_without_a_table_launch_and_the_first_batch_beyond(impl, N):
+    """Up to 16 sequences the intra-chunk kernel finds its chunks from cu_seqlens and writes the
+    per-sequence tables (first chunk, validity, rank) itself; 17 sequences take the table-building
+    launch.  Equal chunk counts (ties in the ranking), an empty sequence, a padding slot and an
+    initial state must come out the same on both sides of that boundary."""
+    lens = [70, 130, 64, 0, 200, 65, 1, 128, 129, 64, 70, 33, 192, 5, 100, 66, 90][:N]
+    p = I.prefill_inputs(lens, 2, 4, seed=900 + N, init="normal")
+    slots = np.arange(N, dtype=np.int32)
+    slots[2] = -1
+    o, S, st = run_prefill(p, impl, slot_idx=slots)
+    assert st == 0
+    o_ref, S_ref, _ = oracle_prefill(p, slot_idx=slots)
+    keep = slots >= 0
+    U.check_o(o, o_ref, U.O_REL_L2_PREFILL)
+    U.check_state(S[keep].astype(np.float64), S_ref[keep], U.STATE_REL_L2_PREFILL)
+    # a batch with out-of-order bounds: flagged, the bad sequence skipped, the others right
+    q = dict(p)
+    cu = p["cu_seqlens"].copy()
+    cu[5] = cu[4] - 3
+    q["cu_seqlens"] = cu
+    _, _, st_bad = run_prefill(q, impl, slot_idx=slots)
+    assert st_bad != 0
