@@ -202,6 +202,8 @@ int gdn_prefill(const void* q, const void* k, const void* v,
  * GDN_RECURRENT_MAX_SEQLEN tokens (by max_seqlen_hint if given, else by the
  * bound T) goes to the token-by-token kernel; anything longer to one of the
  * chunked variants (gdn_prefill_fused for a few long sequence-heads,
+ * gdn_prefill_overlap when max_seqlen_hint tells of chains of at least 32
+ * chunks and there are at most half as many sequence-heads as SMs,
  * gdn_prefill_stream for chains longer than two chunks, more
  * sequence-heads than SMs or at most 16 sequences, else gdn_prefill_chunked).  Each route can also be called directly; arguments
  * are gdn_prefill's.  gdn_prefill_route answers which one gdn_prefill would take
@@ -215,6 +217,7 @@ int gdn_prefill(const void* q, const void* k, const void* v,
 #define GDN_ROUTE_CHUNKED   2
 #define GDN_ROUTE_FUSED     3
 #define GDN_ROUTE_STREAM    4
+#define GDN_ROUTE_OVERLAP   5
 int gdn_prefill_route(int32_t T, int32_t N, int32_t max_seqlen_hint, int32_t Hv,
                       int32_t sm_count, int32_t cooperative_launch);
 int gdn_prefill_chunked(const void* q, const void* k, const void* v,
@@ -258,6 +261,34 @@ int gdn_prefill_stream(const void* q, const void* k, const void* v,
                        int32_t num_slots, float scale,
                        void* workspace, size_t workspace_bytes,
                        int32_t* dev_status, void* stream);
+
+/*
+ * gdn_prefill_overlap - the chunked algorithm (same section of the paper as
+ * gdn_prefill: the prefill regime of the gated delta rule, "through chunked
+ * matrix operations") with the intra-chunk work cut in two around the
+ * persistent state pass: the records the chains need first are produced
+ * before the state pass starts, the others beside it, on the SMs that hold no
+ * live chain, each published through a flag the state pass waits for (bounded
+ * wait; a timeout sets GDN_DEV_TIMEOUT).  For batches of few (sequence,
+ * v-head) units of unequal length.  Arguments, workspace and results are
+ * gdn_prefill_chunked's, plus
+ *   split_permille  share of the (chunk, v-head) items, in the order the
+ *                   chains consume them, produced before the state pass
+ *                   starts: 0..1000, or negative = chosen on the device from
+ *                   the sequence lengths.  With more units than the GPU has
+ *                   SMs to spare everything is produced first (1000).
+ * Four launches on `stream`, programmatic dependents of one another; the call
+ * is complete when the last one is.
+ */
+int gdn_prefill_overlap(const void* q, const void* k, const void* v,
+                        const float* g, const float* beta, const int32_t* cu_seqlens,
+                        const float* init_state, float* final_state, const int32_t* slot_idx,
+                        void* o,
+                        int32_t T, int32_t N, int32_t max_seqlen_hint,
+                        int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv, int32_t chunk,
+                        int32_t num_slots, float scale,
+                        void* workspace, size_t workspace_bytes,
+                        int32_t* dev_status, void* stream, int32_t split_permille);
 
 /*
  * gdn_prefill_recurrent - the same operator and arguments as gdn_prefill,

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libgdn_b200.so")
 
 EXPORTS = ("gdn_decode", "gdn_prefill_workspace_bytes", "gdn_prefill", "gdn_prefill_chunked",
-           "gdn_prefill_fused", "gdn_prefill_stream", "gdn_prefill_route", "gdn_decode_multi", "gdn_gate",
+           "gdn_prefill_fused", "gdn_prefill_stream", "gdn_prefill_overlap", "gdn_prefill_route", "gdn_decode_multi", "gdn_gate",
            "gdn_state_transpose", "gdn_decode_host", "gdn_decode_host_staging_bytes",
            "gdn_prefill_host", "gdn_prefill_host_staging_bytes",
            "gdn_prefill_recurrent",
@@ -55,6 +55,8 @@ _lib.gdn_prefill_route.restype = ctypes.c_int
 _lib.gdn_prefill_route.argtypes = [_I] * 6
 _lib.gdn_prefill_stream.restype = ctypes.c_int
 _lib.gdn_prefill_stream.argtypes = _lib.gdn_prefill.argtypes
+_lib.gdn_prefill_overlap.restype = ctypes.c_int
+_lib.gdn_prefill_overlap.argtypes = _lib.gdn_prefill.argtypes + [_I]
 _lib.gdn_prefill_recurrent.restype = ctypes.c_int
 _lib.gdn_prefill_recurrent.argtypes = [_P] * 10 + [_I] * 7 + [_F, _P, _P]
 _lib.gdn_prefill_static.restype = ctypes.c_int
@@ -164,7 +166,7 @@ def gdn_state_transpose(state_pool, slot_idx=None, n=None, dev_status=None):
         raise GdnError(rc, "gdn_state_transpose")
 
 
-ROUTES = {0: "none", 1: "recurrent", 2: "chunked", 3: "fused", 4: "stream"}
+ROUTES = {0: "none", 1: "recurrent", 2: "chunked", 3: "fused", 4: "stream", 5: "overlap"}
 
 
 def gdn_prefill_route(T, N, max_seqlen_hint, Hv, sm_count=148, cooperative_launch=True) -> str:
@@ -178,16 +180,20 @@ def gdn_prefill_workspace_bytes(T, N, Hqk, Hv, dk=128, dv=128, chunk=64) -> int:
 
 
 def gdn_prefill(q, k, v, g, beta, cu_seqlens, init_state, final_state, slot_idx, o, scale,
-                workspace, max_seqlen_hint=0, chunk=64, dev_status=None, route="auto"):
+                workspace, max_seqlen_hint=0, chunk=64, dev_status=None, route="auto",
+                split_permille=-1):
     """Prefill over packed sequences.  ``workspace`` is a uint8 CUDA tensor.  ``route`` picks the
     entry point: "auto" = gdn_prefill (routes by length), "chunked" = gdn_prefill_chunked (three
     launches), "fused" = gdn_prefill_fused (one cooperative launch), "stream" = gdn_prefill_stream
-    (three launches, persistent state pass)."""
+    (three launches, persistent state pass), "overlap" = gdn_prefill_overlap (the intra-chunk work
+    in two parts around the state pass; ``split_permille`` is its last argument)."""
     T, Hqk, dk = q.shape
     _, Hv, dv = v.shape
     N = cu_seqlens.shape[0] - 1
     fn = {"auto": _lib.gdn_prefill, "chunked": _lib.gdn_prefill_chunked,
-          "fused": _lib.gdn_prefill_fused, "stream": _lib.gdn_prefill_stream}[route]
+          "fused": _lib.gdn_prefill_fused, "stream": _lib.gdn_prefill_stream,
+          "overlap": _lib.gdn_prefill_overlap}[route]
+    extra = (int(split_permille),) if route == "overlap" else ()
     rc = fn(
         _dev(q, torch.bfloat16, "q"), _dev(k, torch.bfloat16, "k"), _dev(v, torch.bfloat16, "v"),
         _dev(g, torch.float32, "g"), _dev(beta, torch.float32, "beta"),
@@ -197,7 +203,7 @@ def gdn_prefill(q, k, v, g, beta, cu_seqlens, init_state, final_state, slot_idx,
         _dev(slot_idx, torch.int32, "slot_idx", True), _dev(o, torch.bfloat16, "o"),
         T, N, int(max_seqlen_hint), Hqk, Hv, dk, dv, int(chunk), final_state.shape[0],
         float(scale), _dev(workspace, torch.uint8, "workspace"), workspace.numel(),
-        _dev(dev_status, torch.int32, "dev_status", True), _stream())
+        _dev(dev_status, torch.int32, "dev_status", True), _stream(), *extra)
     if rc != 0:
         raise GdnError(rc, "gdn_prefill")
 

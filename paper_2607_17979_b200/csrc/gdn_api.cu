@@ -156,14 +156,14 @@ int gdn_prefill_recurrent(const void* q, const void* k, const void* v, const flo
 }
 
 namespace {
-enum PrefillRoute { kRouteChunked, kRouteFused, kRouteStream };
+enum PrefillRoute { kRouteChunked, kRouteFused, kRouteStream, kRouteOverlap };
 
 int prefill_chunked_impl(PrefillRoute route, const void* q, const void* k, const void* v, const float* g,
                          const float* beta, const int32_t* cu_seqlens, const float* init_state,
                          float* final_state, const int32_t* slot_idx, void* o, int32_t T, int32_t N,
                          int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv, int32_t chunk,
                          int32_t num_slots, float scale, void* workspace, size_t workspace_bytes,
-                         int32_t* dev_status, void* stream) {
+                         int32_t* dev_status, void* stream, int32_t split_permille = -1) {
     if (chunk != gdn::kChunk) return GDN_ERR_SHAPE;
     const int rc = check_prefill(q, k, v, g, beta, cu_seqlens, init_state, final_state, o,
                                  T, N, Hqk, Hv, dk, dv, num_slots);
@@ -185,9 +185,10 @@ int prefill_chunked_impl(PrefillRoute route, const void* q, const void* k, const
     cp.ws = static_cast<uint8_t*>(workspace);
     cp.lay = gdn::workspace_layout(T, N, Hv);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    return cuda_status(route == kRouteFused    ? gdn::launch_prefill_fused(cp, st)
-                       : route == kRouteStream ? gdn::launch_prefill_stream(cp, st)
-                                               : gdn::launch_prefill_chunked(cp, st));
+    return cuda_status(route == kRouteFused     ? gdn::launch_prefill_fused(cp, st)
+                       : route == kRouteStream  ? gdn::launch_prefill_stream(cp, st)
+                       : route == kRouteOverlap ? gdn::launch_prefill_overlap(cp, st, split_permille)
+                                                : gdn::launch_prefill_chunked(cp, st));
 }
 }  // namespace
 
@@ -227,6 +228,19 @@ int gdn_prefill_stream(const void* q, const void* k, const void* v, const float*
                                 workspace, workspace_bytes, dev_status, stream);
 }
 
+int gdn_prefill_overlap(const void* q, const void* k, const void* v, const float* g,
+                        const float* beta, const int32_t* cu_seqlens, const float* init_state,
+                        float* final_state, const int32_t* slot_idx, void* o, int32_t T, int32_t N,
+                        int32_t max_seqlen_hint, int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv,
+                        int32_t chunk, int32_t num_slots, float scale, void* workspace,
+                        size_t workspace_bytes, int32_t* dev_status, void* stream,
+                        int32_t split_permille) {
+    (void)max_seqlen_hint;
+    return prefill_chunked_impl(kRouteOverlap, q, k, v, g, beta, cu_seqlens, init_state, final_state,
+                                slot_idx, o, T, N, Hqk, Hv, dk, dv, chunk, num_slots, scale,
+                                workspace, workspace_bytes, dev_status, stream, split_permille);
+}
+
 int gdn_prefill_route(int32_t T, int32_t N, int32_t max_seqlen_hint, int32_t Hv, int32_t sm_count,
                       int32_t cooperative_launch) {
     if (T <= 0 || N <= 0 || Hv <= 0 || sm_count <= 0) return GDN_ROUTE_NONE;
@@ -238,6 +252,16 @@ int gdn_prefill_route(int32_t T, int32_t N, int32_t max_seqlen_hint, int32_t Hv,
     // Few (sequence, v-head) units and long sequences: the serial state pass would occupy only a
     // few SMs while the rest idle, so run it next to the record producers in one cooperative launch.
     if (cooperative_launch && units <= sm_count / 3 && longest > 16 * gdn::kChunk) return GDN_ROUTE_FUSED;
+    // At most half as many units as SMs, with long chains (known only through the caller's hint):
+    // the state pass leaves half the machine free, so part of the records is produced beside it
+    // (measured 10-15 % faster than the three launches on such batches).  Batches that fill the
+    // machine at first and free it as their short chains end gain 5-12 % through
+    // gdn_prefill_overlap too, but the records produced late are still dirty in L2 when the call
+    // ends and their write-back falls into whatever runs next (the next kernel of the varlen
+    // benchmark batch lost half of what the prefill gained), and batches of equal chains lose up
+    // to 7 %: those stay with the persistent state pass.
+    if (max_seqlen_hint > 0 && units <= sm_count / 2 && longest >= 32 * gdn::kChunk)
+        return GDN_ROUTE_OVERLAP;
     // The persistent state pass has the shorter chunk step (its loader, issuer, chain and output
     // warps are separate) and does not pay a CTA start, a pipeline fill and a drain per unit:
     // measured faster whenever a chain is longer than two chunks or there are more units than
@@ -276,9 +300,10 @@ int gdn_prefill(const void* q, const void* k, const void* v, const float* g, con
                                      slot_idx, o, T, N, Hqk, Hv, dk, dv, num_slots, scale,
                                      dev_status, stream);
     }
-    const PrefillRoute route = route_id == GDN_ROUTE_FUSED    ? kRouteFused
-                               : route_id == GDN_ROUTE_STREAM ? kRouteStream
-                                                              : kRouteChunked;
+    const PrefillRoute route = route_id == GDN_ROUTE_FUSED     ? kRouteFused
+                               : route_id == GDN_ROUTE_STREAM  ? kRouteStream
+                               : route_id == GDN_ROUTE_OVERLAP ? kRouteOverlap
+                                                               : kRouteChunked;
     return prefill_chunked_impl(route, q, k, v, g, beta, cu_seqlens, init_state,
                                 final_state, slot_idx, o, T, N, Hqk, Hv, dk, dv, chunk, num_slots,
                                 scale, workspace, workspace_bytes, dev_status, stream);

@@ -54,13 +54,15 @@ struct ChunkInfo {      // 16 bytes
 
 // Workspace layout (all offsets multiples of 256 bytes):
 //   [0,256)                      int32 header: [0] total_chunks, [1] total_items
-//                                (= total_chunks * Hv), [2] item queue head, [3] unit queue head
+//                                (= total_chunks * Hv), [2] item queue head, [3] unit queue head,
+//                                [4] items produced before the state pass starts (two-part route)
 //   seq_first[N+1]               int32: first chunk of each sequence (prefix sum); an invalid
 //                                sequence has zero chunks and seq_bad[n] = 1
 //   seq_bad[N]                   int32
 //   chunks[max_chunks]           ChunkInfo
 //   -- used by the fused single-launch path only --
 //   seq_by_rank[N]               int32: sequences sorted by chunk count, longest first
+//   rank_of[N]                   int32: the inverse (rank of each sequence)
 //   order[max_chunks]            int32: chunk ids in processing order: by position inside the
 //                                sequence first, by sequence rank second (so that the records
 //                                every state-pass unit needs next are produced first)
@@ -69,12 +71,13 @@ struct ChunkInfo {      // 16 bytes
 //   -- both paths --
 //   records[max_chunks][Hv]      kRecBytes each
 struct WorkspaceLayout {
-    size_t seq_first, seq_bad, chunks, seq_by_rank, order, hist, fill, cnt, pos, flags, records,
-        total;
+    size_t seq_first, seq_bad, chunks, seq_by_rank, rank_of, order, hist, fill, cnt, pos, flags,
+        records, total;
     int32_t max_chunks, max_nc;
 };
 
-constexpr int kHdrTotalChunks = 0, kHdrTotalItems = 1, kHdrItemHead = 2, kHdrUnitHead = 3;
+constexpr int kHdrTotalChunks = 0, kHdrTotalItems = 1, kHdrItemHead = 2, kHdrUnitHead = 3,
+              kHdrSplit = 4;
 
 inline size_t round256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 
@@ -88,7 +91,8 @@ inline WorkspaceLayout workspace_layout(int32_t T, int32_t N, int32_t Hv) {
     w.seq_bad = w.seq_first + round256(sizeof(int32_t) * (static_cast<size_t>(N) + 1));
     w.chunks = w.seq_bad + round256(sizeof(int32_t) * static_cast<size_t>(N ? N : 1));
     w.seq_by_rank = w.chunks + round256(sizeof(ChunkInfo) * nchunks);
-    w.order = w.seq_by_rank + round256(sizeof(int32_t) * static_cast<size_t>(N ? N : 1));
+    w.rank_of = w.seq_by_rank + round256(sizeof(int32_t) * static_cast<size_t>(N ? N : 1));
+    w.order = w.rank_of + round256(sizeof(int32_t) * static_cast<size_t>(N ? N : 1));
     w.hist = w.order + round256(sizeof(int32_t) * nchunks);
     w.fill = w.hist + nbins;
     w.cnt = w.fill + nbins;
@@ -114,6 +118,12 @@ cudaError_t launch_prefill_stream(const ChunkedParams& cp, cudaStream_t stream);
 // Pieces shared by the launchers: the prep kernel that also ranks the sequences by chunk count
 // (longest first) and, for the fused launch, orders the chunks and clears the queues and flags;
 // the intra-chunk kernel over all items.
-cudaError_t launch_prefill_ranked_prep(const ChunkedParams& cp, cudaStream_t stream, bool for_fused);
+// mode 0: chunk table and ranking; 1: + processing order, cleared queue heads and flags (fused
+// launch); 2: + the cut of the two-part production (split_permille < 0: the kernel's own model).
+cudaError_t launch_prefill_ranked_prep(const ChunkedParams& cp, cudaStream_t stream, int mode,
+                                       int split_permille = -1, int sms = 0);
+// The intra-chunk kernel in two parts around a flag-gated persistent state pass: the second part
+// of the records is produced beside the chains, on the SMs the state pass leaves free.
+cudaError_t launch_prefill_overlap(const ChunkedParams& cp, cudaStream_t stream, int split_permille);
 
 }  // namespace gdn

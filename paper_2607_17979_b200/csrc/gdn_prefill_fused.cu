@@ -18,11 +18,19 @@ namespace gdn {
 // Prep: chunk table, processing order, cleared queues and flags.  One CTA.
 // =============================================================================================
 constexpr int kFPrepThreads = 256;
+// model of the two-part production (see the kernel): items per SM and chunk step, start-up lag of
+// the second part in chunk steps, and a safety margin in items
+constexpr int kSplitProdPermille = 600;
+constexpr int kSplitLeadSteps = 6;
+constexpr int kSplitMarginItems = 128;
 
 __global__ void __launch_bounds__(kFPrepThreads)
 prefill_fused_prep_kernel(const int32_t* __restrict__ cu, int32_t T, int32_t N, int32_t Hv,
                           uint8_t* ws, WorkspaceLayout lay, int32_t* dev_status,
-                          const int for_fused) {   // 0: only the chunk table and the ranking
+                          const int for_fused,     // 0: only the chunk table and the ranking;
+                                                   // 1: + processing order, cleared queues and flags;
+                                                   // 2: + where the two-part production is cut
+                          const int split_permille, const int sms) {
     int32_t* hdr = reinterpret_cast<int32_t*>(ws);
     int32_t* seq_first = reinterpret_cast<int32_t*>(ws + lay.seq_first);
     int32_t* seq_bad = reinterpret_cast<int32_t*>(ws + lay.seq_bad);
@@ -121,7 +129,7 @@ prefill_fused_prep_kernel(const int32_t* __restrict__ cu, int32_t T, int32_t N, 
     if (tid == 0) running = 0;
     __syncthreads();
     // pos[j] = number of chunks at positions < j: exclusive prefix sum of cnt (fused launch only)
-    for (int base = 0; for_fused && base <= lay.max_nc; base += kFPrepThreads) {
+    for (int base = 0; for_fused != 0 && base <= lay.max_nc; base += kFPrepThreads) {
         const int j = base + tid;
         const int32_t x = j <= lay.max_nc ? cnt[j] : 0;
         int32_t incl = x;
@@ -140,15 +148,58 @@ prefill_fused_prep_kernel(const int32_t* __restrict__ cu, int32_t T, int32_t N, 
         if (tid == kFPrepThreads - 1) running = excl + x;
         __syncthreads();
     }
+    // Two-part production (mode 2).  The items of the processing order before the cut are
+    // produced before the state pass starts, the others beside it, on the SMs it leaves free.
+    // The cut is the smallest head start with which the chains never catch up with the
+    // producers, by a simple model: every live (sequence, v-head) unit consumes one item per
+    // chunk step, the SMs without a live unit produce kProdPermille / 1000 items per chunk step
+    // each, and an item started when the state pass starts is ready kLeadSteps chunk steps
+    // later.  In step j the chains need the Hv * pos[j + 1] first items of the order; by then the
+    // second part has produced r * sum_{i < j - lead} (sms - Hv * cnt[i]), and that sum is
+    // m * sms - Hv * pos[m] with m = j - lead.
+    if (for_fused == 2) {
+        __shared__ int32_t need_max;
+        if (tid == 0) need_max = 0;
+        __syncthreads();
+        const long long total_items = hdr[kHdrTotalItems];
+        long long local = 0;
+        const int lead = kSplitLeadSteps, prod = kSplitProdPermille;
+        for (int j = tid; j < lay.max_nc; j += kFPrepThreads) {
+            const int m = j > lead ? j - lead : 0;
+            long long produced =
+                (static_cast<long long>(m) * sms - static_cast<long long>(Hv) * pos[m]) * prod / 1000;
+            if (produced < 0) produced = 0;
+            const long long need = static_cast<long long>(Hv) * pos[j + 1] - produced;
+            local = need > local ? need : local;
+        }
+        if (local > total_items) local = total_items;
+        atomicMax(&need_max, static_cast<int32_t>(local));
+        __syncthreads();
+        if (tid == 0) {
+            long long cut = split_permille >= 0 ? total_items * split_permille / 1000
+                                                : static_cast<long long>(need_max) + kSplitMarginItems;
+            if (cut > total_items) cut = total_items;
+            hdr[kHdrSplit] = static_cast<int32_t>(cut);
+        }
+    }
     // rank of a sequence = its place in the order "more chunks first"; chunk j of the sequence of
     // rank r is processed at place pos[j] + r (the sequences that have a chunk j are ranks < cnt[j])
+    int32_t* rank_of = reinterpret_cast<int32_t*>(ws + lay.rank_of);
     for (int n = tid; n < N; n += kFPrepThreads) {
         const int32_t nc = seq_first[n + 1] - seq_first[n];
         const int32_t rank = cnt[nc] + atomicAdd(&fill[nc], 1);
         seq_by_rank[rank] = n;
-        const int32_t first = seq_first[n];
-        if (for_fused)
-            for (int j = 0; j < nc; ++j) order[pos[j] + rank] = first + j;
+        rank_of[n] = rank;
+    }
+    if (for_fused) {
+        // one thread per chunk (a loop per sequence would be a chain of dependent loads as long
+        // as the longest sequence)
+        __syncthreads();
+        const int32_t total_chunks = hdr[kHdrTotalChunks];
+        for (int c = tid; c < total_chunks; c += kFPrepThreads) {
+            const int32_t n = chunks[c].seq;
+            order[pos[c - seq_first[n]] + rank_of[n]] = c;
+        }
     }
 }
 
@@ -238,7 +289,7 @@ prefill_fused_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
     tc_fence_after_sync();
     const uint32_t tmem = tmem_base_s;
     if (static_cast<int>(blockIdx.x) < n_state) {
-        state_stream_role<true>(maps, p, ws, lay, smem, tmem, blockIdx.x, n_state);
+        state_stream_role<1>(maps, p, ws, lay, smem, tmem, blockIdx.x, n_state);
     } else {
         fused_intra_role(maps, p, ws, lay, smem, intra_statics, tmem);
         tc_fence_before_sync();
@@ -250,10 +301,11 @@ prefill_fused_kernel(const __grid_constant__ TensorMaps maps, const PrefillParam
 // =============================================================================================
 // host side
 // =============================================================================================
-cudaError_t launch_prefill_ranked_prep(const ChunkedParams& cp, cudaStream_t stream, bool for_fused) {
+cudaError_t launch_prefill_ranked_prep(const ChunkedParams& cp, cudaStream_t stream, int mode,
+                                       int split_permille, int sms) {
     prefill_fused_prep_kernel<<<1, kFPrepThreads, 0, stream>>>(cp.p.cu_seqlens, cp.p.T, cp.p.N,
                                                                cp.p.Hv, cp.ws, cp.lay,
-                                                               cp.p.dev_status, for_fused ? 1 : 0);
+                                                               cp.p.dev_status, mode, split_permille, sms);
     return cudaGetLastError();
 }
 
@@ -271,7 +323,7 @@ cudaError_t launch_prefill_fused(const ChunkedParams& cp, cudaStream_t stream) {
     TensorMaps maps;
     if (!make_prefill_tensor_maps(&maps, p)) return cudaErrorInvalidValue;
 
-    e = launch_prefill_ranked_prep(cp, stream, true);
+    e = launch_prefill_ranked_prep(cp, stream, 1);
     if (e != cudaSuccess) return e;
 
     // How many CTAs run the state pass: one per unit when the units are few (the shapes routed

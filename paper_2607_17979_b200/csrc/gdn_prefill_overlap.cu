@@ -1,0 +1,189 @@
+// Chunked prefill with the record production in two parts around the persistent state pass.
+//
+// With few (sequence, v-head) units of unequal length the state pass is a handful of long serial
+// chains: most SMs hold a short chain that ends early, or none, while the intra-chunk kernel
+// before it needs the whole machine.  Here the intra-chunk work is cut in two along the order in
+// which the chains consume the records (by position inside the sequence first): the first part
+// runs alone, then the state pass starts, one CTA per unit, and the second part runs beside it on
+// the SMs that have no live chain, each record published through a flag (release) that the state
+// pass's loading warp waits for (acquire, bounded).
+//
+// Four launches in one stream, each a programmatic dependent of the one before:
+//   prep          chunk table, ranking, processing order, cleared flags, the cut
+//   first part    waits for prep; items [0, cut) of the order, 4 CTAs per SM
+//   state pass    waits for the first part, THEN lets its dependent start, so the second part's
+//                 CTAs are scheduled only once every state-pass CTA is resident: they can never
+//                 take the SMs the chains need, and every chain that waits for a record is
+//                 resident while the producers still have SMs of their own (the launcher keeps
+//                 units <= SMs - kOverlapSpareSms)
+//   second part   does not wait for the state pass (it only feeds it); items [cut, total), pulled
+//                 from a queue by at most four CTAs per SM.  Its
+//                 CTA 0 waits for the state pass at its very end, so that the completion of this
+//                 last launch implies the completion of the whole call.
+#include "gdn_prefill_stream.cuh"
+
+namespace gdn {
+
+constexpr int kOverlapSpareSms = 8;
+
+// First part: one CTA per item [0, cut) of the processing order (surplus CTAs exit).
+__global__ void __launch_bounds__(kIntraThreads, 4)
+prefill_intra_first_kernel(const __grid_constant__ TensorMaps maps, const PrefillParams p,
+                           uint8_t* ws, const WorkspaceLayout lay) {
+    pdl_launch_dependents();
+    pdl_wait();                     // the tables are the prep kernel's
+    const int32_t* hdr = reinterpret_cast<const int32_t*>(ws);
+    const int item = blockIdx.x;
+    if (item >= hdr[kHdrSplit]) return;
+    const int k = item / p.Hv;
+    const int hv = item - k * p.Hv;
+    const int c = reinterpret_cast<const int32_t*>(ws + lay.order)[k];
+    const ChunkInfo ci = reinterpret_cast<const ChunkInfo*>(ws + lay.chunks)[c];
+    uint8_t* rec = ws + lay.records + (static_cast<size_t>(c) * p.Hv + hv) * kRecBytes;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                               ~static_cast<uintptr_t>(1023));
+    __shared__ IntraStatics st;
+    __shared__ uint32_t tmem_base_s;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    if (warp == 0) {
+        tmem_alloc(&tmem_base_s, kIntraTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = tmem_base_s;
+    intra_item(maps, p, rec, ci, hv / (p.Hv / p.Hqk), hv, smem, st, tmem, tid, [] { __syncthreads(); });
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, kIntraTmemCols);
+}
+
+// Second part: resident CTAs pull the items [cut, total) from a queue, in the order the chains
+// consume them, and publish each record through its flag.  No wait for the state pass (this kernel
+// feeds it): every state-pass CTA has passed its own wait for the first part, hence for prep,
+// before this kernel's CTAs are scheduled.
+__global__ void __launch_bounds__(kIntraThreads, 4)
+prefill_intra_second_kernel(const __grid_constant__ TensorMaps maps, const PrefillParams p,
+                            uint8_t* ws, const WorkspaceLayout lay) {
+    int32_t* hdr = reinterpret_cast<int32_t*>(ws);
+    const int32_t cut = hdr[kHdrSplit], total = hdr[kHdrTotalItems];
+    const int32_t* order = reinterpret_cast<const int32_t*>(ws + lay.order);
+    const ChunkInfo* chunks = reinterpret_cast<const ChunkInfo*>(ws + lay.chunks);
+    uint32_t* flags = reinterpret_cast<uint32_t*>(ws + lay.flags);
+    const int G = p.Hv / p.Hqk;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                               ~static_cast<uintptr_t>(1023));
+    __shared__ IntraStatics st;
+    __shared__ uint32_t tmem_base_s;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    if (cut < total) {
+        if (warp == 0) {
+            tmem_alloc(&tmem_base_s, kIntraTmemCols);
+            tmem_relinquish();
+        }
+        tc_fence_before_sync();
+        __syncthreads();
+        tc_fence_after_sync();
+        const uint32_t tmem = tmem_base_s;
+        uint32_t n_done = 0;
+        for (;;) {
+            if (tid == 0) st.item = cut + atomicAdd(&hdr[kHdrItemHead], 1);
+            __syncthreads();
+            const int item = st.item;
+            if (item >= total) break;
+            const int k = item / p.Hv;
+            const int hv = item - k * p.Hv;
+            const int c = order[k];
+            const ChunkInfo ci = chunks[c];
+            const size_t slot = static_cast<size_t>(c) * p.Hv + hv;
+            uint8_t* rec = ws + lay.records + slot * kRecBytes;
+            const bool ok = intra_item(maps, p, rec, ci, hv / G, hv, smem, st, tmem, tid,
+                                       [] { __syncthreads(); }, n_done);
+            ++n_done;
+            // publish: every thread's own stores first, then the bulk stores, then the flag
+            __threadfence();
+            tc_fence_before_sync();
+            __syncthreads();
+            if (tid == 0) {
+                bulk_wait_all();
+                fence_proxy_async_all();
+                __threadfence();
+                st_release_u32(&flags[slot], ok ? 1u : 2u);      // 2 = produced after a timeout
+            }
+            if (!ok) break;
+        }
+        tc_fence_before_sync();
+        __syncthreads();
+        if (warp == 0) tmem_dealloc(tmem, kIntraTmemCols);
+    }
+    if (blockIdx.x == 0) pdl_wait();        // the call is complete when this launch is
+}
+
+__global__ void __launch_bounds__(kStreamThreads, 1)
+prefill_state_stream_gated_kernel(const __grid_constant__ TensorMaps maps, const PrefillParams p,
+                                  uint8_t* ws, const WorkspaceLayout lay) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                               ~static_cast<uintptr_t>(1023));
+    __shared__ uint32_t tmem_base_s;
+    const int warp = threadIdx.x >> 5;
+    if (warp == kSIssueWarp) {
+        tmem_alloc(&tmem_base_s, kStateTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = tmem_base_s;
+    pdl_wait();                     // tables, cleared flags and the first part's records
+    pdl_launch_dependents();        // now the second part may take the SMs that are left
+    state_stream_role<2>(maps, p, ws, lay, smem, tmem, blockIdx.x, gridDim.x);
+    __syncwarp();
+    if (warp == kSIssueWarp) tmem_dealloc(tmem, kStateTmemCols);
+}
+
+cudaError_t launch_prefill_overlap(const ChunkedParams& cp, cudaStream_t stream, int split_permille) {
+    const PrefillParams& p = cp.p;
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    e = cudaFuncSetAttribute(prefill_state_stream_gated_kernel,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(prefill_intra_first_kernel,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, kIntraSmem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(prefill_intra_second_kernel,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, kIntraSmem);
+    if (e != cudaSuccess) return e;
+    TensorMaps maps;
+    if (!make_prefill_tensor_maps(&maps, p)) return cudaErrorInvalidValue;
+
+    // The second part needs SMs of its own for as long as a chain may wait for it: with (nearly)
+    // as many units as SMs everything is produced before the state pass starts.
+    const long long units = static_cast<long long>(p.N) * p.Hv;
+    if (units > sms - kOverlapSpareSms) split_permille = 1000;
+    if (split_permille > 1000) split_permille = 1000;
+
+    e = launch_prefill_ranked_prep(cp, stream, 2, split_permille, sms);
+    if (e != cudaSuccess) return e;
+    const dim3 items(static_cast<unsigned>(cp.lay.max_chunks) * static_cast<unsigned>(p.Hv));
+    e = launch_dependent(prefill_intra_first_kernel, items, dim3(kIntraThreads), kIntraSmem,
+                         stream, maps, p, cp.ws, cp.lay);
+    if (e != cudaSuccess) return e;
+    const int grid = static_cast<int>(units < sms ? units : sms);
+    e = launch_dependent(prefill_state_stream_gated_kernel, dim3(grid), dim3(kStreamThreads),
+                         kStreamSmem, stream, maps, p, cp.ws, cp.lay);
+    if (e != cudaSuccess) return e;
+    const unsigned resident = 4u * static_cast<unsigned>(sms);
+    return launch_dependent(prefill_intra_second_kernel, dim3(items.x < resident ? items.x : resident),
+                            dim3(kIntraThreads), kIntraSmem, stream, maps, p, cp.ws, cp.lay);
+}
+
+}  // namespace gdn

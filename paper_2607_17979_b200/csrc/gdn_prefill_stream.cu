@@ -20,7 +20,7 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = tmem_base_s;
-    state_stream_role<false>(maps, p, ws, lay, smem, tmem, blockIdx.x, gridDim.x);
+    state_stream_role<0>(maps, p, ws, lay, smem, tmem, blockIdx.x, gridDim.x);
     __syncwarp();
     if (warp == kSIssueWarp) tmem_dealloc(tmem, kStateTmemCols);
 }
@@ -40,7 +40,7 @@ cudaError_t launch_prefill_stream(const ChunkedParams& cp, cudaStream_t stream) 
     if (!make_prefill_tensor_maps(&maps, p)) return cudaErrorInvalidValue;
     const bool inline_tables = prefill_tables_inline(cp);
     if (!inline_tables) {
-        e = launch_prefill_ranked_prep(cp, stream, false);
+        e = launch_prefill_ranked_prep(cp, stream, 0);
         if (e != cudaSuccess) return e;
     }
     if (cp.lay.max_chunks > 0) {

@@ -87,10 +87,12 @@ __device__ __forceinline__ void fence_proxy_async_all() {
 }
 
 // The state pass of one CTA of 512 threads over the units cta, cta + n_ctas, ... of the rank-sorted
-// list.  kGated = false: every record exists (the intra-chunk kernel ran before).  kGated = true:
+// list.  kGated = 0: every record exists (the intra-chunk kernel ran before).  kGated = 1:
 // records are being produced by other CTAs of the same cooperative launch and the loading warp
-// waits for each record's flag first.  `tmem` = 512 allocated columns; ends with a CTA barrier.
-template <bool kGated>
+// waits for each record's flag first.  kGated = 2: the records of the first hdr[kHdrSplit] items of
+// the processing order exist, the others are being produced by a concurrent kernel and are waited
+// for.  `tmem` = 512 allocated columns; ends with a CTA barrier.
+template <int kGated>
 __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const PrefillParams& p,
                                                   uint8_t* ws, const WorkspaceLayout& lay,
                                                   uint8_t* smem, const uint32_t tmem, const int cta,
@@ -135,7 +137,7 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
     __syncthreads();
     tc_fence_after_sync();
     volatile int* abortp = &abort_flag;
-    if constexpr (!kGated) pdl_wait();     // tables and records are the previous kernels'
+    if constexpr (kGated == 0) pdl_wait();     // tables and records are the previous kernels'
 
     // gc = chunks of earlier units of this CTA; chunk j of the current unit is chunk g = gc + j of
     // the CTA's stream: stage g & 1, phase g >> 1 of bar_full / bar_free_* of that stage, phase g of
@@ -156,6 +158,12 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
             const uint32_t* flags = reinterpret_cast<const uint32_t*>(ws + lay.flags);
             (void)flags;
             bool live = true;
+            // kGated == 2: chunk j of the sequence of rank r is item (pos[j] + r) * Hv + hv of
+            // the processing order; items from `cut` on are waited for
+            const int32_t* pos = reinterpret_cast<const int32_t*>(ws + lay.pos);
+            const int32_t cut = kGated == 2 ? reinterpret_cast<const int32_t*>(ws)[kHdrSplit] : 0;
+            (void)pos;
+            (void)cut;
             // the next unit's table entries are fetched while the current unit is processed
             UnitInfo nxt = unit_info(p, ws, lay, min(cta, total_units - 1));
             for (int unit = cta; unit < total_units && live; unit += n_ctas) {
@@ -164,6 +172,8 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
                 if (u.skip) continue;
                 const uint8_t* records =
                     ws + lay.records + (static_cast<size_t>(u.c_first) * p.Hv + u.hv) * kRecBytes;
+                const int32_t rank = unit / p.Hv;
+                int32_t pos_j = kGated == 2 ? pos[0] : 0;       // fetched one chunk ahead
                 for (int j = 0; j < u.nc; ++j) {
                     const uint32_t g = gc + j;
                     const int st = g & 1;
@@ -171,7 +181,12 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
                     const uint32_t par_free = ((g - 2) >> 1) & 1u;
                     uint8_t* base = smem + st * kStageBytes;
                     const uint8_t* rec = records + j * rec_stride;
-                    if constexpr (kGated) {
+                    bool gated = kGated == 1;
+                    if constexpr (kGated == 2) {
+                        gated = (pos_j + rank) * p.Hv + u.hv >= cut;
+                        pos_j = pos[j + 1];                     // pos has an entry past the longest chain
+                    }
+                    if (gated) {
                         // the record must have been published by its producer CTA
                         const uint32_t* f = flags + (static_cast<size_t>(u.c_first + j) * p.Hv + u.hv);
                         uint32_t v = 0;

@@ -9,11 +9,11 @@ import gpu_util as U
 
 pytestmark = pytest.mark.gpu
 
-IMPLS = ["chunked", "fused", "stream", "recurrent"]
+IMPLS = ["chunked", "fused", "stream", "overlap", "recurrent"]
 
 
 def run_prefill(p, impl, slot_idx=None, num_slots=None, init="from_inputs", alias=False,
-                pool_fill=None):
+                pool_fill=None, split_permille=-1):
     """Returns (o fp64 [T,Hv,128], final fp32 numpy [num_slots,Hv,128,128], status)."""
     from paper_2607_17979_b200 import api
     N, Hv, T = p["N"], p["Hv"], p["T"]
@@ -30,10 +30,10 @@ def run_prefill(p, impl, slot_idx=None, num_slots=None, init="from_inputs", alia
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     args = (U.dev_bf16(p["q"]), U.dev_bf16(p["k"]), U.dev_bf16(p["v"]), U.dev(p["g"]),
             U.dev(p["beta"]), U.dev(p["cu_seqlens"]), init_t, final, U.dev(slot_idx), o, p["scale"])
-    if impl in ("chunked", "fused", "stream", "auto"):
+    if impl in ("chunked", "fused", "stream", "overlap", "auto"):
         ws = torch.empty(max(api.gdn_prefill_workspace_bytes(T, N, p["Hqk"], Hv), 256),
                          dtype=torch.uint8, device="cuda")
-        api.gdn_prefill(*args, ws, dev_status=status, route=impl)
+        api.gdn_prefill(*args, ws, dev_status=status, route=impl, split_permille=split_permille)
     else:
         api.gdn_prefill_recurrent(*args, dev_status=status)
     torch.cuda.synchronize()
@@ -191,7 +191,7 @@ def test_prefill_long_context_benchmark_config_sampled_heads():
             U.check_state(S[:, hv:hv + 1].astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
 
 
-@pytest.mark.parametrize("impl", ["auto", "chunked", "stream", "fused"])
+@pytest.mark.parametrize("impl", ["auto", "chunked", "stream", "fused", "overlap"])
 def test_batches_that_are_all_padding_or_all_empty(impl):
     """No valid work at all: every slot negative (rows zeroed, no state touched), and every
     sequence but one empty (states pass through bit-exactly)."""
@@ -220,7 +220,7 @@ def test_thousands_of_tiny_sequences():
         U.check_state(S.astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
 
 
-@pytest.mark.parametrize("impl", ["chunked", "stream", "fused"])
+@pytest.mark.parametrize("impl", ["chunked", "stream", "fused", "overlap"])
 def test_chunked_repeatable_under_load_many_ctas(impl):
     """Several back-to-back runs of a batch that fills the GPU (64 sequence-heads, ragged tails,
     last chunks of every length class) must be bit-identical: a missed barrier between the
@@ -298,3 +298,42 @@ def test_small_batches_without_a_table_launch_and_the_first_batch_beyond(impl, N
     q["cu_seqlens"] = cu
     _, _, st_bad = run_prefill(q, impl, slot_idx=slots)
     assert st_bad != 0
+
+
+@pytest.mark.parametrize("split", [-1, 0, 150, 400, 1000])
+def test_two_part_production_at_any_cut(split):
+    """gdn_prefill_overlap produces the records before the cut ahead of the state pass and the
+    others beside it, behind flags: every cut (none, some, all of the items up front, or the
+    library's own choice) must give the oracle's result, with sequences of very unequal length,
+    an empty one, a padding slot and a ragged tail in the batch."""
+    lens = [1500, 64, 0, 333, 700, 1]
+    p = I.prefill_inputs(lens, 2, 4, seed=77, init="normal")
+    num_slots = 8
+    slots = np.array([5, 0, 3, -1, 7, 2], np.int32)
+    init = np.zeros((num_slots, 4, 128, 128), np.float32)
+    for n in range(len(lens)):
+        if slots[n] >= 0:
+            init[slots[n]] = p["init_state"][n]
+    o_ref, S_ref, _ = oracle.prefill(p["q"], p["k"], p["v"], p["g"], p["beta"], p["cu_seqlens"],
+                                     init.astype(np.float64), slots, p["scale"], num_slots=num_slots)
+    o, S, status = run_prefill(p, "overlap", slot_idx=slots, num_slots=num_slots, init=init,
+                               pool_fill=0.0, split_permille=split)
+    assert status == 0
+    U.check_o(o, o_ref, U.O_REL_L2_PREFILL)
+    keep = slots[slots >= 0]
+    U.check_state(S[keep].astype(np.float64), S_ref[keep], U.STATE_REL_L2_PREFILL)
+    untouched = [s for s in range(num_slots) if s not in keep]
+    assert np.array_equal(S[untouched], init[untouched])
+
+
+def test_two_part_production_matches_the_three_launches_bit_for_bit():
+    """Same kernels' arithmetic in another schedule: on the varlen benchmark shape the overlapped
+    route and the persistent state pass must agree exactly, whatever the cut."""
+    from paper_2607_17979_b200 import api
+    p = I.prefill_inputs([512, 1024, 2048, 4096], 16, 32, seed=5, init="zero")
+    o_s, S_s, st_s = run_prefill(p, "stream", init=None)
+    for split in (-1, 300):
+        o_o, S_o, st_o = run_prefill(p, "overlap", init=None, split_permille=split)
+        assert st_s == 0 and st_o == 0
+        assert np.array_equal(o_s, o_o) and np.array_equal(S_s, S_o)
+    assert api.gdn_prefill_route(8192, 2, 4096, 32) == "overlap"
