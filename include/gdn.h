@@ -202,7 +202,7 @@ int gdn_prefill(const void* q, const void* k, const void* v,
  * GDN_RECURRENT_MAX_SEQLEN tokens (by max_seqlen_hint if given, else by the
  * bound T) goes to the token-by-token kernel; anything longer to one of the
  * chunked variants (gdn_prefill_fused for a few long sequence-heads,
- * gdn_prefill_overlap when max_seqlen_hint tells of chains of at least 32
+ * gdn_prefill_overlap when max_seqlen_hint tells of chains of at least 40
  * chunks and there are at most half as many sequence-heads as SMs,
  * gdn_prefill_stream for chains longer than two chunks, more
  * sequence-heads than SMs or at most 16 sequences, else gdn_prefill_chunked).  Each route can also be called directly; arguments

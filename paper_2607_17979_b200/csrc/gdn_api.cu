@@ -254,13 +254,14 @@ int gdn_prefill_route(int32_t T, int32_t N, int32_t max_seqlen_hint, int32_t Hv,
     if (cooperative_launch && units <= sm_count / 3 && longest > 16 * gdn::kChunk) return GDN_ROUTE_FUSED;
     // At most half as many units as SMs, with long chains (known only through the caller's hint):
     // the state pass leaves half the machine free, so part of the records is produced beside it
-    // (measured 10-15 % faster than the three launches on such batches).  Batches that fill the
+    // (measured 10-15 % faster than the three launches on such batches from about 40 chunks on;
+    // two chains of 32 chunks were 4 % slower).  Batches that fill the
     // machine at first and free it as their short chains end gain 5-12 % through
     // gdn_prefill_overlap too, but the records produced late are still dirty in L2 when the call
     // ends and their write-back falls into whatever runs next (the next kernel of the varlen
     // benchmark batch lost half of what the prefill gained), and batches of equal chains lose up
     // to 7 %: those stay with the persistent state pass.
-    if (max_seqlen_hint > 0 && units <= sm_count / 2 && longest >= 32 * gdn::kChunk)
+    if (max_seqlen_hint > 0 && units <= sm_count / 2 && longest >= 40 * gdn::kChunk)
         return GDN_ROUTE_OVERLAP;
     // The persistent state pass has the shorter chunk step (its loader, issuer, chain and output
     // warps are separate) and does not pay a CTA start, a pipeline fill and a drain per unit:
