@@ -95,7 +95,7 @@ def main():
     ap.add_argument("--reps", type=int, default=200)
     ap.add_argument("--lens", default="", help="time one prefill shape only: comma-separated "
                     "sequence lengths, LENxCOUNT for repeats (e.g. 144x56,128)")
-    ap.add_argument("--route", default="auto", choices=["auto", "chunked", "fused", "stream"])
+    ap.add_argument("--route", default="auto", choices=["auto", "chunked", "fused", "stream", "overlap"])
     ap.add_argument("--decode-multi", default="", help="time one multi-token decode shape only: "
                     "BxL (both state orientations)")
     args = ap.parse_args()
