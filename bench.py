@@ -39,6 +39,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures
 # (profiles/); None until a capture of that kernel exists.
 NCU_TRAFFIC_BYTES = {"decode": 213_381_376, "prefill": 730_488_832}
+# one dependent chunk step of the persistent state pass (clock stamps in a debug build: about 3630
+# cycles at 1965 MHz); the serial bound of a prefill call is the longest chain times this
+CHUNK_STEP_US = 1.85
 
 
 def peaks():
@@ -275,15 +278,17 @@ def run_ours(args):
         dec_ms = np.array([a.elapsed_time(b) for a, b, _, _ in evs])
         pre_ms = np.array([c.elapsed_time(d) for _, _, c, d in evs])
         slowest = D.max_over_ranks([dec_ms.mean(), pre_ms.mean()], device="cuda")
-        return slowest[0], slowest[1]
+        spread = {"decode_ms_median": float(np.median(dec_ms)), "decode_ms_min": float(dec_ms.min()),
+                  "prefill_ms_median": float(np.median(pre_ms)), "prefill_ms_min": float(pre_ms.min())}
+        return slowest[0], slowest[1], spread
 
     # clocks are sampled from before the warm-up to after the timed steps (the GPU is under the
     # same load throughout; the timed steps alone can be shorter than one sampling period)
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    dec_ms, pre_ms = timed_region(step)
-    e2e_dec_ms, e2e_pre_ms = timed_region(e2e_step)
+    dec_ms, pre_ms, spread = timed_region(step)
+    e2e_dec_ms, e2e_pre_ms, _ = timed_region(e2e_step)
     clocks = sampler.stop() if rank == 0 else None
     assert int(status.item()) == 0, "device status flagged during the benchmark"
 
@@ -312,7 +317,8 @@ def run_ours(args):
                        "l2": f"inputs larger than L2: decode rotates over {DEC_POOLS} distinct 128 MiB "
                              f"state pools (1 GiB), prefill over {PRE_SETS} distinct input sets "
                              "(3 x 190 MB) plus its workspace",
-                       "decode_ms": dec_ms, "prefill_ms": pre_ms},
+                       "decode_ms": dec_ms, "prefill_ms": pre_ms,
+                       "this_rank_spread": spread},
             "roofline": {"kernel": "gdn decode", "bound": "hbm", "achieved": dec_ach,
                          "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": dec_ach / pk["hbm_gbs"],
                          "peak_kind": pk_kind, "frac_of_nominal_8TBps": dec_ach / 8000.0,
@@ -326,6 +332,11 @@ def run_ours(args):
                                      "frac_of_roofline_time": pre_roof_ms / pre_ms,
                                      "algorithmic_bytes": pre_b, "algorithmic_flops": pre_f,
                                      "traffic": NCU_TRAFFIC_BYTES["prefill"]},
+                        # the serial part: the longest sequence's chunks, one dependent chunk step
+                        # each (step time from a cycle trace of the state pass, not from this run)
+                        "chain_bound": {"depth_chunks": -(-max(pre["seq_lens"]) // 64),
+                                        "chunk_step_us": CHUNK_STEP_US,
+                                        "ms": -(-max(pre["seq_lens"]) // 64) * CHUNK_STEP_US * 1e-3},
                         "e2e": {"value": world * T / (e2e_pre_ms * 1e-3), "unit": "tokens/s",
                                 "h2d_bytes_per_step": h2d_p,
                                 "d2h_bytes_per_step": h_po.numel() * 2},

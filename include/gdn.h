@@ -278,7 +278,11 @@ int gdn_prefill_stream(const void* q, const void* k, const void* v,
  *                   the sequence lengths.  With more units than the GPU has
  *                   SMs to spare everything is produced first (1000).
  * Four launches on `stream`, programmatic dependents of one another; the call
- * is complete when the last one is.
+ * is complete when the last one is.  The state pass waits for records of the
+ * launch behind it, so the two must be able to run concurrently: with
+ * CUDA_LAUNCH_BLOCKING set everything is produced first; under a tool that
+ * replays kernels one at a time the bounded waits run out (GDN_DEV_TIMEOUT, no
+ * hang) - profile gdn_prefill_stream there.
  */
 int gdn_prefill_overlap(const void* q, const void* k, const void* v,
                         const float* g, const float* beta, const int32_t* cu_seqlens,

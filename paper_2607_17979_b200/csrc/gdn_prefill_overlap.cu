@@ -21,6 +21,7 @@
 //                 CTA 0 waits for the state pass at its very end, so that the completion of this
 //                 last launch implies the completion of the whole call.
 #include "gdn_prefill_stream.cuh"
+#include <cstdlib>
 
 namespace gdn {
 
@@ -169,6 +170,13 @@ cudaError_t launch_prefill_overlap(const ChunkedParams& cp, cudaStream_t stream,
     // as many units as SMs everything is produced before the state pass starts.
     const long long units = static_cast<long long>(p.N) * p.Hv;
     if (units > sms - kOverlapSpareSms) split_permille = 1000;
+    // The state pass waits for a launch that comes after it in the stream: the two must be able to
+    // run at the same time.  Where launches are known to be serialised, produce everything first
+    // (then no record is waited for).  A profiler that replays kernels one at a time cannot be
+    // seen from here: under it the waits run out (GDN_DEV_TIMEOUT, no hang); profile
+    // gdn_prefill_stream instead, which runs the same kernels' arithmetic.
+    const char* blocking = std::getenv("CUDA_LAUNCH_BLOCKING");
+    if (blocking && blocking[0] != '\0' && blocking[0] != '0') split_permille = 1000;
     if (split_permille > 1000) split_permille = 1000;
 
     e = launch_prefill_ranked_prep(cp, stream, 2, split_permille, sms);

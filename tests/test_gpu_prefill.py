@@ -156,13 +156,15 @@ def test_chunked_and_recurrent_routes_agree():
     assert U.rel_l2(Sc.astype(np.float64), Sr.astype(np.float64)) <= U.STATE_REL_L2_PREFILL
 
 
-def test_prefill_varlen_benchmark_config_full():
-    """4 sequences {512,1024,2048,4096}, 32 v-heads: every output against the oracle, through the
-    length-routed entry point (the call the benchmark times) and through the plain three launches."""
-    p = I.make_config(3, 0)
+@pytest.mark.parametrize("trial", [0, 1, 2])
+def test_prefill_varlen_benchmark_config_full(trial):
+    """4 sequences {512,1024,2048,4096}, 32 v-heads, three seeds: every output against the oracle,
+    through the length-routed entry point (the call the benchmark times) and, on the first seed,
+    through the plain three launches and the two-part production."""
+    p = I.make_config(3, trial)
     o_ref, S_ref, _ = oracle_prefill(p)
     cu = p["cu_seqlens"]
-    for impl in ("auto", "chunked"):
+    for impl in (("auto", "chunked", "overlap") if trial == 0 else ("auto",)):
         o, S, status = run_prefill(p, impl)
         assert status == 0
         U.check_o(o, o_ref, U.O_REL_L2_PREFILL)
@@ -171,18 +173,20 @@ def test_prefill_varlen_benchmark_config_full():
             U.check_o(o[cu[n]:cu[n + 1]], o_ref[cu[n]:cu[n + 1]], U.O_REL_L2_PREFILL)
 
 
-def test_prefill_long_context_benchmark_config_sampled_heads():
+@pytest.mark.parametrize("trial", [0, 1])
+def test_prefill_long_context_benchmark_config_sampled_heads(trial):
     """One 32768-token sequence at full size on the GPU, through the length-routed entry point
-    (the fused launch for this shape) and the plain three launches; the oracle recomputes four
-    sampled v-heads (each with its own q/k head) over the whole sequence."""
-    p = I.make_config(4, 0)
+    (the fused launch for this shape) and the plain three launches (first seed) or the two-part
+    production (second seed); the oracle recomputes four sampled v-heads (each with its own q/k
+    head) over the whole sequence."""
+    p = I.make_config(4, trial)
     refs = {}
     for hv in (0, 13, 22, 31):
         hq = hv // 2
         refs[hv] = oracle.prefill(p["q"][:, hq:hq + 1], p["k"][:, hq:hq + 1], p["v"][:, hv:hv + 1],
                                   p["g"][:, hv:hv + 1], p["beta"][:, hv:hv + 1], p["cu_seqlens"],
                                   p["init_state"][:, hv:hv + 1].astype(np.float64), None, p["scale"])
-    for impl in ("auto", "chunked"):
+    for impl in (("auto", "chunked") if trial == 0 else ("auto", "overlap")):
         o, S, status = run_prefill(p, impl)
         assert status == 0 and np.isfinite(o).all() and np.isfinite(S).all()
         for hv, (o_ref, S_ref, _) in refs.items():
