@@ -341,3 +341,43 @@ def test_two_part_production_matches_the_three_launches_bit_for_bit():
         assert st_s == 0 and st_o == 0
         assert np.array_equal(o_s, o_o) and np.array_equal(S_s, S_o)
     assert api.gdn_prefill_route(8192, 2, 4096, 32) == "overlap"
+
+
+def test_two_part_production_replayed_from_a_cuda_graph():
+    """The four launches are programmatic dependents of one another and the last does not wait for
+    the one before it; captured into a CUDA graph and replayed they must still give the eager
+    result (the flags and the queue are cleared by the first launch of every call)."""
+    from paper_2607_17979_b200 import api
+    p = I.prefill_inputs([2600, 700, 65], 2, 4, seed=9, init="zero")
+    T, N = p["T"], p["N"]
+    ws = torch.empty(api.gdn_prefill_workspace_bytes(T, N, 2, 4), dtype=torch.uint8, device="cuda")
+    args = (U.dev_bf16(p["q"]), U.dev_bf16(p["k"]), U.dev_bf16(p["v"]), U.dev(p["g"]),
+            U.dev(p["beta"]), U.dev(p["cu_seqlens"]))
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def outs():
+        return (torch.zeros((N, 4, 128, 128), dtype=torch.float32, device="cuda"),
+                torch.zeros((T, 4, 128), dtype=torch.bfloat16, device="cuda"))
+
+    f0, o0 = outs()
+    api.gdn_prefill(*args, None, f0, None, o0, p["scale"], ws, route="overlap", split_permille=300,
+                    dev_status=status)
+    torch.cuda.synchronize()
+    f1, o1 = outs()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for _ in range(2):
+                api.gdn_prefill(*args, None, f1, None, o1, p["scale"], ws, route="overlap",
+                                split_permille=300, dev_status=status)
+    for _ in range(3):
+        f1.zero_()
+        o1.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(f0, f1) and torch.equal(o0, o1)
+    assert int(status.item()) == 0
+    o_ref, S_ref, _ = oracle_prefill(p, init=None)
+    U.check_o(U.host_f64_from_bf16(o1), o_ref, U.O_REL_L2_PREFILL)
+    U.check_state(f1.cpu().numpy().astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
