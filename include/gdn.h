@@ -201,9 +201,10 @@ int gdn_prefill(const void* q, const void* k, const void* v,
  * gdn_prefill routes by shape: a batch whose longest sequence has at most
  * GDN_RECURRENT_MAX_SEQLEN tokens (by max_seqlen_hint if given, else by the
  * bound T) goes to the token-by-token kernel; anything longer to one of the
- * chunked variants (gdn_prefill_fused for a few long sequence-heads,
- * gdn_prefill_overlap when max_seqlen_hint tells of chains of at least 40
- * chunks and there are at most half as many sequence-heads as SMs,
+ * chunked variants (gdn_prefill_overlap when max_seqlen_hint tells of chains
+ * of at least 40 chunks and there are at most half as many sequence-heads as
+ * SMs, gdn_prefill_fused for a single long sequence of few heads and for
+ * few long sequence-heads without such a hint,
  * gdn_prefill_stream for chains longer than two chunks, more
  * sequence-heads than SMs or at most 16 sequences, else gdn_prefill_chunked).  Each route can also be called directly; arguments
  * are gdn_prefill's.  gdn_prefill_route answers which one gdn_prefill would take
