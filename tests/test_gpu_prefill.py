@@ -242,7 +242,7 @@ def test_chunked_repeatable_under_load_many_ctas(impl):
     U.check_state(ref_S.astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
 
 
-@pytest.mark.parametrize("impl", ["stream", "auto"])
+@pytest.mark.parametrize("impl", ["stream", "auto", "overlap"])
 def test_many_short_sequences_stream_across_unit_boundaries(impl):
     """Far more (sequence, v-head) units than SMs, of mixed lengths (one to five chunks, ragged
     tails, empty sequences, a padding slot): every CTA of the persistent state pass walks a
