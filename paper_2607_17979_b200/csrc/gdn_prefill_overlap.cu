@@ -17,7 +17,7 @@
 //                 resident while the producers still have SMs of their own (the launcher keeps
 //                 units <= SMs - kOverlapSpareSms)
 //   second part   does not wait for the state pass (it only feeds it); items [cut, total), pulled
-//                 from a queue by at most four CTAs per SM.  Its
+//                 from a queue by seven CTAs per unit (at most four per SM).  Its
 //                 CTA 0 waits for the state pass at its very end, so that the completion of this
 //                 last launch implies the completion of the whole call.
 #include "gdn_prefill_stream.cuh"
