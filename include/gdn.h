@@ -201,10 +201,7 @@ int gdn_prefill(const void* q, const void* k, const void* v,
  * gdn_prefill routes by shape: a batch whose longest sequence has at most
  * GDN_RECURRENT_MAX_SEQLEN tokens (by max_seqlen_hint if given, else by the
  * bound T) goes to the token-by-token kernel; anything longer to one of the
- * chunked variants (gdn_prefill_overlap when max_seqlen_hint tells of chains
- * of at least 40 chunks and there are at most half as many sequence-heads as
- * SMs, gdn_prefill_fused for a single long sequence of few heads and for
- * few long sequence-heads without such a hint,
+ * chunked variants (gdn_prefill_fused for a few long sequence-heads,
  * gdn_prefill_stream for chains longer than two chunks, more
  * sequence-heads than SMs or at most 16 sequences, else gdn_prefill_chunked).  Each route can also be called directly; arguments
  * are gdn_prefill's.  gdn_prefill_route answers which one gdn_prefill would take
@@ -218,7 +215,6 @@ int gdn_prefill(const void* q, const void* k, const void* v,
 #define GDN_ROUTE_CHUNKED   2
 #define GDN_ROUTE_FUSED     3
 #define GDN_ROUTE_STREAM    4
-#define GDN_ROUTE_OVERLAP   5
 int gdn_prefill_route(int32_t T, int32_t N, int32_t max_seqlen_hint, int32_t Hv,
                       int32_t sm_count, int32_t cooperative_launch);
 int gdn_prefill_chunked(const void* q, const void* k, const void* v,
@@ -279,8 +275,12 @@ int gdn_prefill_stream(const void* q, const void* k, const void* v,
  *                   the sequence lengths.  With more units than the GPU has
  *                   SMs to spare everything is produced first (1000).
  * Four launches on `stream`, programmatic dependents of one another; the call
- * is complete when the last one is.  The state pass waits for records of the
- * launch behind it, so the two must be able to run concurrently: with
+ * is complete when the last one is.  gdn_prefill never chooses this route by
+ * itself (it is not among gdn_prefill_route's answers): the
+ * state pass waits for records of the launch behind it, so the two must run
+ * at the same time, which programmatic dependent launch makes the device do
+ * but which CUDA does not promise.  If it does not happen the bounded waits
+ * run out and GDN_DEV_TIMEOUT is set (results invalid, no hang).  With
  * CUDA_LAUNCH_BLOCKING set everything is produced first; under a tool that
  * replays kernels one at a time the bounded waits run out (GDN_DEV_TIMEOUT, no
  * hang) - profile gdn_prefill_stream there.

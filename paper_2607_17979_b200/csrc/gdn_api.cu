@@ -249,25 +249,14 @@ int gdn_prefill_route(int32_t T, int32_t N, int32_t max_seqlen_hint, int32_t Hv,
     // very short sequences: the token-by-token kernel (one launch, no workspace traffic)
     if (longest <= GDN_RECURRENT_MAX_SEQLEN) return GDN_ROUTE_RECURRENT;
     const long long units = static_cast<long long>(N) * Hv;
-    // At most half as many units as SMs, with long chains (known only through the caller's hint):
-    // the state pass leaves half the machine free from the start, so part of the records is
-    // produced beside it, by a kernel of four CTAs per SM on the free SMs (measured 10-15 % faster
-    // than the three launches on such batches from about 40 chunks on; two chains of 32 chunks
-    // were 4 % slower).  Batches that fill the machine at first and free it as their short chains
-    // end gain 5-12 % through gdn_prefill_overlap too, but the records produced late are still
-    // dirty in L2 when the call ends and their write-back falls into whatever runs next (the
-    // next kernel of the varlen benchmark batch lost half of what the prefill gained), and
-    // batches of equal chains lose up to 7 %: those stay with the persistent state pass.
-    const bool overlap_ok =
-        max_seqlen_hint > 0 && units <= sm_count / 2 && longest >= 40 * gdn::kChunk;
-    // Few units and long sequences: the producers run beside the state pass in one cooperative
-    // launch.  Against the two-part production it is level for a single sequence (ahead by 5 % at
-    // 32768 tokens) and behind by 2-20 % for several (its producers run two items per SM, and
-    // with 48 units it was slower than the three launches), so it keeps the single sequences and
-    // the batches the two-part production does not take.
-    const bool fused_ok = cooperative_launch && units <= sm_count / 3 && longest > 16 * gdn::kChunk;
-    if (fused_ok && (N == 1 || !overlap_ok)) return GDN_ROUTE_FUSED;
-    if (overlap_ok) return GDN_ROUTE_OVERLAP;
+    // Few (sequence, v-head) units and long sequences: the serial state pass would occupy only a
+    // few SMs while the rest idle, so run it next to the record producers in one cooperative launch.
+    if (cooperative_launch && units <= sm_count / 3 && longest > 16 * gdn::kChunk) return GDN_ROUTE_FUSED;
+    // gdn_prefill_overlap is never chosen here although it is the fastest route for long chains
+    // on at most half the SMs (10-15 % ahead of the three launches, 2-20 % ahead of the
+    // cooperative launch for several sequences): its state pass waits for a later launch, and
+    // that the two run at the same time is what the device does, not what CUDA promises.  The
+    // cooperative launch gives that promise; a caller who accepts the other asks for it by name.
     // The persistent state pass has the shorter chunk step (its loader, issuer, chain and output
     // warps are separate) and does not pay a CTA start, a pipeline fill and a drain per unit:
     // measured faster whenever a chain is longer than two chunks or there are more units than
@@ -308,7 +297,6 @@ int gdn_prefill(const void* q, const void* k, const void* v, const float* g, con
     }
     const PrefillRoute route = route_id == GDN_ROUTE_FUSED     ? kRouteFused
                                : route_id == GDN_ROUTE_STREAM  ? kRouteStream
-                               : route_id == GDN_ROUTE_OVERLAP ? kRouteOverlap
                                                                : kRouteChunked;
     return prefill_chunked_impl(route, q, k, v, g, beta, cu_seqlens, init_state,
                                 final_state, slot_idx, o, T, N, Hqk, Hv, dk, dv, chunk, num_slots,

@@ -120,15 +120,9 @@ def test_prefill_routing_rules_are_pure_host_arithmetic():
     assert r(1600, 16, 100, 4) == "stream" and r(1700, 17, 100, 4) == "chunked"
     assert r(8192, 128, 64, 32) == "stream" and r(296, 37, 8, 4) != "stream"        # 4096 / 148 units
     assert r(1184, 37, 32, 4) == "chunked" and r(1216, 38, 32, 4) == "stream"       # 148 / 152 units
-    # the caller says how long the longest sequence is, chains of at least 40 chunks and at most
-    # half as many units as SMs: part of the records is produced beside the state pass
-    assert r(8192, 2, 4096, 32) == "overlap" and r(4000, 2, 3000, 32) == "overlap"
-    assert r(8192, 2, 0, 32) == "stream" and r(5118, 2, 2559, 32) == "stream"
-    assert r(7680, 4, 4096, 32) == "stream" and r(6144, 3, 2048, 32) == "stream"    # 128 / 96 units
-    assert r(8192, 2, 4096, 37) == "overlap" and r(8192, 2, 4096, 38) == "stream"   # 74 / 76 units
-    # few units: several sequences with a hint go the same way, a single sequence (or no hint)
-    # to the cooperative launch
-    assert r(8192, 2, 4096, 8) == "overlap" and r(8192, 2, 0, 8) == "fused"
-    assert r(4096, 1, 4096, 32) == "fused" and r(4000, 2, 2000, 8) == "fused"
+    # the two-part production (its state pass waits for a later launch) is never chosen
+    # automatically, whatever the hint
+    assert r(8192, 2, 4096, 32) == "stream" and r(8192, 2, 4096, 8) == "fused"
+    assert r(7680, 4, 4096, 32) == "stream" and r(6144, 3, 2048, 32) == "stream"
     # the thresholds follow the SM count given
     assert r(1184, 37, 32, 4, 100) == "stream"
