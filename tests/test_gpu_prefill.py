@@ -9,7 +9,7 @@ import gpu_util as U
 
 pytestmark = pytest.mark.gpu
 
-IMPLS = ["chunked", "fused", "stream", "overlap", "recurrent"]
+IMPLS = ["chunked", "fused", "stream", "recurrent"]
 
 
 def run_prefill(p, impl, slot_idx=None, num_slots=None, init="from_inputs", alias=False,
@@ -160,11 +160,11 @@ def test_chunked_and_recurrent_routes_agree():
 def test_prefill_varlen_benchmark_config_full(trial):
     """4 sequences {512,1024,2048,4096}, 32 v-heads, three seeds: every output against the oracle,
     through the length-routed entry point (the call the benchmark times) and, on the first seed,
-    through the plain three launches and the two-part production."""
+    through the plain three launches."""
     p = I.make_config(3, trial)
     o_ref, S_ref, _ = oracle_prefill(p)
     cu = p["cu_seqlens"]
-    for impl in (("auto", "chunked", "overlap") if trial == 0 else ("auto",)):
+    for impl in (("auto", "chunked") if trial == 0 else ("auto",)):
         o, S, status = run_prefill(p, impl)
         assert status == 0
         U.check_o(o, o_ref, U.O_REL_L2_PREFILL)
@@ -176,8 +176,7 @@ def test_prefill_varlen_benchmark_config_full(trial):
 @pytest.mark.parametrize("trial", [0, 1])
 def test_prefill_long_context_benchmark_config_sampled_heads(trial):
     """One 32768-token sequence at full size on the GPU, through the length-routed entry point
-    (the fused launch for this shape) and the plain three launches (first seed) or the two-part
-    production (second seed); the oracle recomputes four sampled v-heads (each with its own q/k
+    (the fused launch for this shape) and, on the first seed, the plain three launches; the oracle recomputes four sampled v-heads (each with its own q/k
     head) over the whole sequence."""
     p = I.make_config(4, trial)
     refs = {}
@@ -186,7 +185,7 @@ def test_prefill_long_context_benchmark_config_sampled_heads(trial):
         refs[hv] = oracle.prefill(p["q"][:, hq:hq + 1], p["k"][:, hq:hq + 1], p["v"][:, hv:hv + 1],
                                   p["g"][:, hv:hv + 1], p["beta"][:, hv:hv + 1], p["cu_seqlens"],
                                   p["init_state"][:, hv:hv + 1].astype(np.float64), None, p["scale"])
-    for impl in (("auto", "chunked") if trial == 0 else ("auto", "overlap")):
+    for impl in (("auto", "chunked") if trial == 0 else ("auto",)):
         o, S, status = run_prefill(p, impl)
         assert status == 0 and np.isfinite(o).all() and np.isfinite(S).all()
         for hv, (o_ref, S_ref, _) in refs.items():
@@ -195,7 +194,7 @@ def test_prefill_long_context_benchmark_config_sampled_heads(trial):
             U.check_state(S[:, hv:hv + 1].astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
 
 
-@pytest.mark.parametrize("impl", ["auto", "chunked", "stream", "fused", "overlap"])
+@pytest.mark.parametrize("impl", ["auto", "chunked", "stream", "fused"])
 def test_batches_that_are_all_padding_or_all_empty(impl):
     """No valid work at all: every slot negative (rows zeroed, no state touched), and every
     sequence but one empty (states pass through bit-exactly)."""
@@ -224,7 +223,7 @@ def test_thousands_of_tiny_sequences():
         U.check_state(S.astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
 
 
-@pytest.mark.parametrize("impl", ["chunked", "stream", "fused", "overlap"])
+@pytest.mark.parametrize("impl", ["chunked", "stream", "fused"])
 def test_chunked_repeatable_under_load_many_ctas(impl):
     """Several back-to-back runs of a batch that fills the GPU (64 sequence-heads, ragged tails,
     last chunks of every length class) must be bit-identical: a missed barrier between the
@@ -242,7 +241,7 @@ def test_chunked_repeatable_under_load_many_ctas(impl):
     U.check_state(ref_S.astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
 
 
-@pytest.mark.parametrize("impl", ["stream", "auto", "overlap"])
+@pytest.mark.parametrize("impl", ["stream", "auto"])
 def test_many_short_sequences_stream_across_unit_boundaries(impl):
     """Far more (sequence, v-head) units than SMs, of mixed lengths (one to five chunks, ragged
     tails, empty sequences, a padding slot): every CTA of the persistent state pass walks a
@@ -302,81 +301,4 @@ def test_small_batches_without_a_table_launch_and_the_first_batch_beyond(impl, N
     q["cu_seqlens"] = cu
     _, _, st_bad = run_prefill(q, impl, slot_idx=slots)
     assert st_bad != 0
-
-
-@pytest.mark.parametrize("split", [-1, 0, 150, 400, 1000])
-def test_two_part_production_at_any_cut(split):
-    """gdn_prefill_overlap produces the records before the cut ahead of the state pass and the
-    others beside it, behind flags: every cut (none, some, all of the items up front, or the
-    library's own choice) must give the oracle's result, with sequences of very unequal length,
-    an empty one, a padding slot and a ragged tail in the batch."""
-    lens = [1500, 64, 0, 333, 700, 1]
-    p = I.prefill_inputs(lens, 2, 4, seed=77, init="normal")
-    num_slots = 8
-    slots = np.array([5, 0, 3, -1, 7, 2], np.int32)
-    init = np.zeros((num_slots, 4, 128, 128), np.float32)
-    for n in range(len(lens)):
-        if slots[n] >= 0:
-            init[slots[n]] = p["init_state"][n]
-    o_ref, S_ref, _ = oracle.prefill(p["q"], p["k"], p["v"], p["g"], p["beta"], p["cu_seqlens"],
-                                     init.astype(np.float64), slots, p["scale"], num_slots=num_slots)
-    o, S, status = run_prefill(p, "overlap", slot_idx=slots, num_slots=num_slots, init=init,
-                               pool_fill=0.0, split_permille=split)
-    assert status == 0
-    U.check_o(o, o_ref, U.O_REL_L2_PREFILL)
-    keep = slots[slots >= 0]
-    U.check_state(S[keep].astype(np.float64), S_ref[keep], U.STATE_REL_L2_PREFILL)
-    untouched = [s for s in range(num_slots) if s not in keep]
-    assert np.array_equal(S[untouched], init[untouched])
-
-
-def test_two_part_production_matches_the_three_launches_bit_for_bit():
-    """Same kernels' arithmetic in another schedule: on the varlen benchmark shape the overlapped
-    route and the persistent state pass must agree exactly, whatever the cut."""
-    p = I.prefill_inputs([512, 1024, 2048, 4096], 16, 32, seed=5, init="zero")
-    o_s, S_s, st_s = run_prefill(p, "stream", init=None)
-    for split in (-1, 300):
-        o_o, S_o, st_o = run_prefill(p, "overlap", init=None, split_permille=split)
-        assert st_s == 0 and st_o == 0
-        assert np.array_equal(o_s, o_o) and np.array_equal(S_s, S_o)
-
-
-def test_two_part_production_replayed_from_a_cuda_graph():
-    """The four launches are programmatic dependents of one another and the last does not wait for
-    the one before it; captured into a CUDA graph and replayed they must still give the eager
-    result (the flags and the queue are cleared by the first launch of every call)."""
-    from paper_2607_17979_b200 import api
-    p = I.prefill_inputs([2600, 700, 65], 2, 4, seed=9, init="zero")
-    T, N = p["T"], p["N"]
-    ws = torch.empty(api.gdn_prefill_workspace_bytes(T, N, 2, 4), dtype=torch.uint8, device="cuda")
-    args = (U.dev_bf16(p["q"]), U.dev_bf16(p["k"]), U.dev_bf16(p["v"]), U.dev(p["g"]),
-            U.dev(p["beta"]), U.dev(p["cu_seqlens"]))
-    status = torch.zeros(1, dtype=torch.int32, device="cuda")
-
-    def outs():
-        return (torch.zeros((N, 4, 128, 128), dtype=torch.float32, device="cuda"),
-                torch.zeros((T, 4, 128), dtype=torch.bfloat16, device="cuda"))
-
-    f0, o0 = outs()
-    api.gdn_prefill(*args, None, f0, None, o0, p["scale"], ws, route="overlap", split_permille=300,
-                    dev_status=status)
-    torch.cuda.synchronize()
-    f1, o1 = outs()
-    side = torch.cuda.Stream()
-    with torch.cuda.stream(side):
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=side):
-            for _ in range(2):
-                api.gdn_prefill(*args, None, f1, None, o1, p["scale"], ws, route="overlap",
-                                split_permille=300, dev_status=status)
-    for _ in range(3):
-        f1.zero_()
-        o1.zero_()
-        graph.replay()
-        torch.cuda.synchronize()
-        assert torch.equal(f0, f1) and torch.equal(o0, o1)
-    assert int(status.item()) == 0
-    o_ref, S_ref, _ = oracle_prefill(p, init=None)
-    U.check_o(U.host_f64_from_bf16(o1), o_ref, U.O_REL_L2_PREFILL)
-    U.check_state(f1.cpu().numpy().astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
 

@@ -35,7 +35,7 @@ def test_random_batch_all_routes(seed):
     o_ref, S_ref, _ = oracle.prefill(p["q"], p["k"], p["v"], p["g"], p["beta"], p["cu_seqlens"],
                                      init.astype(np.float64), slots, p["scale"], num_slots=num_slots)
     keep = slots[slots >= 0]
-    for impl in ("chunked", "fused", "stream", "overlap", "recurrent", "auto"):
+    for impl in ("chunked", "fused", "stream", "recurrent", "auto"):
         o, S, status = run_prefill(p, impl, slot_idx=slots, num_slots=num_slots, init=init,
                                    pool_fill=0.0)
         assert status == 0, impl
