@@ -266,7 +266,7 @@ int gdn_prefill_stream(const void* q, const void* k, const void* v,
  * persistent state pass: the records the chains need first are produced
  * before the state pass starts, the others beside it, on the SMs that hold no
  * live chain, each published through a flag the state pass waits for (bounded
- * wait; a timeout sets GDN_DEV_TIMEOUT).  For batches of few (sequence,
+ * wait).  For batches of few (sequence,
  * v-head) units of unequal length.  Arguments, workspace and results are
  * gdn_prefill_chunked's, plus
  *   split_permille  share of the (chunk, v-head) items, in the order the
@@ -274,16 +274,19 @@ int gdn_prefill_stream(const void* q, const void* k, const void* v,
  *                   starts: 0..1000, or negative = chosen on the device from
  *                   the sequence lengths.  With more units than the GPU has
  *                   SMs to spare everything is produced first (1000).
- * Four launches on `stream`, programmatic dependents of one another; the call
- * is complete when the last one is.  gdn_prefill never chooses this route by
- * itself (it is not among gdn_prefill_route's answers): the
- * state pass waits for records of the launch behind it, so the two must run
+ *                   -2 = as negative, but the producers of the second part
+ *                   are launched as an ordinary successor of the state pass
+ *                   (serialised on purpose: the recovery path, for tests).
+ * Five launches on `stream`; the call is complete when the last one is.  The
+ * state pass waits for records of the launch behind it, so the two should run
  * at the same time, which programmatic dependent launch makes the device do
- * but which CUDA does not promise.  If it does not happen the bounded waits
- * run out and GDN_DEV_TIMEOUT is set (results invalid, no hang).  With
- * CUDA_LAUNCH_BLOCKING set everything is produced first; under a tool that
- * replays kernels one at a time the bounded waits run out (GDN_DEV_TIMEOUT, no
- * hang) - profile gdn_prefill_stream there.
+ * but which CUDA does not promise (and a tool that replays kernels one at a
+ * time prevents).  If it does not happen the waits for records run out after
+ * a fraction of a second, the state pass marks the (sequence, v-head) units it
+ * has finished and the last launch runs the others once the records exist:
+ * the results are the same, only time is lost.  For that reason gdn_prefill
+ * never chooses this route by itself (it is not among gdn_prefill_route's
+ * answers).  With CUDA_LAUNCH_BLOCKING set everything is produced first.
  */
 int gdn_prefill_overlap(const void* q, const void* k, const void* v,
                         const float* g, const float* beta, const int32_t* cu_seqlens,

@@ -68,11 +68,13 @@ struct ChunkInfo {      // 16 bytes
 //                                every state-pass unit needs next are produced first)
 //   hist, fill, cnt, pos[max_nc+2]  int32 scratch of the counting sort (max_nc = T/64 + 1)
 //   flags[max_chunks][Hv]        uint32: 1 once the record is complete and visible
+//   done[N][Hv]                  int32: 1 once the two-part route's state pass has finished the unit
+//                                (rank-major, like the unit list); the rest is left to a last launch
 //   -- both paths --
 //   records[max_chunks][Hv]      kRecBytes each
 struct WorkspaceLayout {
     size_t seq_first, seq_bad, chunks, seq_by_rank, rank_of, order, hist, fill, cnt, pos, flags,
-        records, total;
+        done, records, total;
     int32_t max_chunks, max_nc;
 };
 
@@ -98,7 +100,8 @@ inline WorkspaceLayout workspace_layout(int32_t T, int32_t N, int32_t Hv) {
     w.cnt = w.fill + nbins;
     w.pos = w.cnt + nbins;
     w.flags = w.pos + nbins;
-    w.records = w.flags + round256(sizeof(uint32_t) * nchunks * Hv);
+    w.done = w.flags + round256(sizeof(uint32_t) * nchunks * Hv);
+    w.records = w.done + round256(sizeof(int32_t) * static_cast<size_t>(N ? N : 1) * Hv);
     w.total = w.records + static_cast<size_t>(w.max_chunks) * Hv * kRecBytes;
     return w;
 }

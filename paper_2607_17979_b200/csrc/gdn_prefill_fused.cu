@@ -51,6 +51,10 @@ prefill_fused_prep_kernel(const int32_t* __restrict__ cu, int32_t T, int32_t N, 
     if (for_fused)
         for (size_t i = tid; i < static_cast<size_t>(lay.max_chunks) * Hv; i += kFPrepThreads)
             flags[i] = 0u;
+    if (for_fused == 2) {
+        int32_t* done = reinterpret_cast<int32_t*>(ws + lay.done);
+        for (int i = tid; i < N * Hv; i += kFPrepThreads) done[i] = 0;
+    }
     if (tid == 0) {
         running = 0;
         hdr[kHdrItemHead] = 0;

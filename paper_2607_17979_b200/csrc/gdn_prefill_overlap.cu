@@ -8,18 +8,25 @@
 // the SMs that have no live chain, each record published through a flag (release) that the state
 // pass's loading warp waits for (acquire, bounded).
 //
-// Four launches in one stream, each a programmatic dependent of the one before:
-//   prep          chunk table, ranking, processing order, cleared flags, the cut
+// Five launches in one stream, the first four each a programmatic dependent of the one before:
+//   prep          chunk table, ranking, processing order, cleared flags and done table, the cut
 //   first part    waits for prep; items [0, cut) of the order, 4 CTAs per SM
 //   state pass    waits for the first part, THEN lets its dependent start, so the second part's
 //                 CTAs are scheduled only once every state-pass CTA is resident: they can never
 //                 take the SMs the chains need, and every chain that waits for a record is
 //                 resident while the producers still have SMs of their own (the launcher keeps
-//                 units <= SMs - kOverlapSpareSms)
+//                 units <= SMs - kOverlapSpareSms, so every CTA has one unit)
 //   second part   does not wait for the state pass (it only feeds it); items [cut, total), pulled
-//                 from a queue by seven CTAs per unit (at most four per SM).  Its
-//                 CTA 0 waits for the state pass at its very end, so that the completion of this
-//                 last launch implies the completion of the whole call.
+//                 from a queue by seven CTAs per unit (at most four per SM).  Its CTA 0 waits
+//                 for the state pass at its very end, so that the completion of this launch
+//                 implies the state pass's.
+//   rest          an ordinary launch.  CUDA lets a programmatic dependent start early, it does not
+//                 promise to; if the second part did not run beside the state pass, the state
+//                 pass's waits for records ran out (soon, and without an error: a unit's final
+//                 state is written only after its last record has been loaded, so an unfinished
+//                 unit has left its initial state alone), it marked the units it finished, and
+//                 this launch runs the persistent pass over the others now that every record
+//                 exists.  Normally every CTA finds its unit done and returns at once.
 #include "gdn_prefill_stream.cuh"
 #include <cstdlib>
 
@@ -148,6 +155,37 @@ prefill_state_stream_gated_kernel(const __grid_constant__ TensorMaps maps, const
     if (warp == kSIssueWarp) tmem_dealloc(tmem, kStateTmemCols);
 }
 
+// Last launch: the plain persistent pass over the units the gated pass did not finish (none, when
+// the producers ran beside it as intended: then every CTA finds its units done and returns).
+__global__ void __launch_bounds__(kStreamThreads, 1)
+prefill_state_stream_rest_kernel(const __grid_constant__ TensorMaps maps, const PrefillParams p,
+                                 uint8_t* ws, const WorkspaceLayout lay) {
+    // nothing left for this CTA: leave before any set-up
+    {
+        const int32_t* done = reinterpret_cast<const int32_t*>(ws + lay.done);
+        const int total_units = p.N * p.Hv;
+        bool any = false;
+        for (int unit = blockIdx.x; unit < total_units; unit += gridDim.x) any = any || done[unit] == 0;
+        if (!any) return;
+    }
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                               ~static_cast<uintptr_t>(1023));
+    __shared__ uint32_t tmem_base_s;
+    const int warp = threadIdx.x >> 5;
+    if (warp == kSIssueWarp) {
+        tmem_alloc(&tmem_base_s, kStateTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = tmem_base_s;
+    state_stream_role<3>(maps, p, ws, lay, smem, tmem, blockIdx.x, gridDim.x);
+    __syncwarp();
+    if (warp == kSIssueWarp) tmem_dealloc(tmem, kStateTmemCols);
+}
+
 cudaError_t launch_prefill_overlap(const ChunkedParams& cp, cudaStream_t stream, int split_permille) {
     const PrefillParams& p = cp.p;
     int dev = 0, sms = 0;
@@ -155,6 +193,9 @@ cudaError_t launch_prefill_overlap(const ChunkedParams& cp, cudaStream_t stream,
     if (e != cudaSuccess) return e;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     e = cudaFuncSetAttribute(prefill_state_stream_gated_kernel,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(prefill_state_stream_rest_kernel,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmem);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(prefill_intra_first_kernel,
@@ -168,6 +209,9 @@ cudaError_t launch_prefill_overlap(const ChunkedParams& cp, cudaStream_t stream,
 
     // The second part needs SMs of its own for as long as a chain may wait for it: with (nearly)
     // as many units as SMs everything is produced before the state pass starts.
+    // split_permille == -2 (for tests): the second part is launched as an ordinary successor of
+    // the state pass, i.e. the launches are serialised on purpose
+    const bool serialised = split_permille == -2;
     const long long units = static_cast<long long>(p.N) * p.Hv;
     if (units > sms - kOverlapSpareSms) split_permille = 1000;
     // The state pass waits for a launch that comes after it in the stream: the two must be able to
@@ -196,8 +240,19 @@ cudaError_t launch_prefill_overlap(const ChunkedParams& cp, cudaStream_t stream,
     unsigned resident = 7u * static_cast<unsigned>(units);
     if (resident < static_cast<unsigned>(sms)) resident = static_cast<unsigned>(sms);
     if (resident > 4u * static_cast<unsigned>(sms)) resident = 4u * static_cast<unsigned>(sms);
-    return launch_dependent(prefill_intra_second_kernel, dim3(items.x < resident ? items.x : resident),
-                            dim3(kIntraThreads), kIntraSmem, stream, maps, p, cp.ws, cp.lay);
+    const dim3 producers(items.x < resident ? items.x : resident);
+    if (serialised) {
+        prefill_intra_second_kernel<<<producers, kIntraThreads, kIntraSmem, stream>>>(maps, p, cp.ws, cp.lay);
+        e = cudaGetLastError();
+    } else {
+        e = launch_dependent(prefill_intra_second_kernel, producers, dim3(kIntraThreads), kIntraSmem,
+                             stream, maps, p, cp.ws, cp.lay);
+    }
+    if (e != cudaSuccess) return e;
+    // an ordinary launch: it starts when the second part has ended, and the second part's first
+    // CTA ends only after the state pass
+    prefill_state_stream_rest_kernel<<<grid, kStreamThreads, kStreamSmem, stream>>>(maps, p, cp.ws, cp.lay);
+    return cudaGetLastError();
 }
 
 }  // namespace gdn

@@ -49,10 +49,12 @@ struct UnitInfo {
     int n, hv, hqk, c_first, nc, seq_t0, seq_len, slot;
     bool skip;          // invalid sequence, padding / out-of-range slot, or no chunks
     bool bad_seq, bad_slot;
+    bool done;          // finished by an earlier launch (the two-part route's last launch only)
 };
 
 __device__ __forceinline__ UnitInfo unit_info(const PrefillParams& p, const uint8_t* ws,
-                                              const WorkspaceLayout& lay, int unit) {
+                                              const WorkspaceLayout& lay, int unit,
+                                              const int32_t* done = nullptr) {   // units to leave out
     const int32_t* seq_first = reinterpret_cast<const int32_t*>(ws + lay.seq_first);
     const int32_t* seq_bad = reinterpret_cast<const int32_t*>(ws + lay.seq_bad);
     const int32_t* seq_by_rank = reinterpret_cast<const int32_t*>(ws + lay.seq_by_rank);
@@ -69,10 +71,12 @@ __device__ __forceinline__ UnitInfo unit_info(const PrefillParams& p, const uint
     u.bad_seq = seq_bad[u.n] != 0;
     u.bad_slot = u.slot < 0 || u.slot >= p.num_slots;
     u.skip = u.bad_seq || u.bad_slot || u.nc == 0;
+    u.done = done != nullptr && done[unit] != 0;
     return u;
 }
 
 constexpr uint32_t kSpinFlagLimit = 1u << 22;
+constexpr uint32_t kSpinFlagLimitSoft = 1u << 17;
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
     uint32_t v;
@@ -91,7 +95,10 @@ __device__ __forceinline__ void fence_proxy_async_all() {
 // records are being produced by other CTAs of the same cooperative launch and the loading warp
 // waits for each record's flag first.  kGated = 2: the records of the first hdr[kHdrSplit] items of
 // the processing order exist, the others are being produced by a concurrent kernel and are waited
-// for.  `tmem` = 512 allocated columns; ends with a CTA barrier.
+// for; a wait that runs out ends the CTA's work without an error (the units it has finished are
+// marked in the done table, the others are left to a later launch).  kGated = 3: that later launch:
+// every record exists, the units marked done are left out.  `tmem` = 512 allocated columns; ends
+// with a CTA barrier.
 template <int kGated>
 __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const PrefillParams& p,
                                                   uint8_t* ws, const WorkspaceLayout& lay,
@@ -105,6 +112,9 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
     const int dv = (warp & 3) * 32 + lane;            // TMEM lane = state row
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const int total_units = p.N * p.Hv;
+    int32_t* done_w = reinterpret_cast<int32_t*>(ws + lay.done);      // written by kGated == 2
+    const int32_t* done_tab = kGated == 3 ? done_w : nullptr;         // read by kGated == 3
+    (void)done_w;
 
     if (tid == 0) {
         mbar_init(&bar_full[0], 1);
@@ -165,11 +175,11 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
             (void)pos;
             (void)cut;
             // the next unit's table entries are fetched while the current unit is processed
-            UnitInfo nxt = unit_info(p, ws, lay, min(cta, total_units - 1));
+            UnitInfo nxt = unit_info(p, ws, lay, min(cta, total_units - 1), done_tab);
             for (int unit = cta; unit < total_units && live; unit += n_ctas) {
                 const UnitInfo u = nxt;
-                nxt = unit_info(p, ws, lay, min(unit + n_ctas, total_units - 1));
-                if (u.skip) continue;
+                nxt = unit_info(p, ws, lay, min(unit + n_ctas, total_units - 1), done_tab);
+                if (u.skip || u.done) continue;
                 const uint8_t* records =
                     ws + lay.records + (static_cast<size_t>(u.c_first) * p.Hv + u.hv) * kRecBytes;
                 const int32_t rank = unit / p.Hv;
@@ -190,12 +200,20 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
                         // the record must have been published by its producer CTA
                         const uint32_t* f = flags + (static_cast<size_t>(u.c_first + j) * p.Hv + u.hv);
                         uint32_t v = 0;
-                        for (uint32_t i = 0; i < kSpinFlagLimit; ++i) {
+                        // kGated == 2: a wait that runs out is no error (the producers' launch may
+                        // not be running beside this one): give up soon, well before any of the
+                        // other roles' waits, and leave the unit to the last launch
+                        const uint32_t limit = kGated == 2 ? kSpinFlagLimitSoft : kSpinFlagLimit;
+                        for (uint32_t i = 0; i < limit; ++i) {
                             v = ld_acquire_u32(f);
                             if (v != 0 || *abortp) break;
                             __nanosleep(64);
                         }
-                        if (v != 1) { *abortp = 1; live = false; break; }
+                        if (v != 1) {
+                            if (*abortp == 0) *abortp = (kGated == 2 && v == 0) ? 2 : 1;
+                            live = false;
+                            break;
+                        }
                         // No proxy fence here: the producer put one between its generic stores and
                         // the flag's release, which is on the path from those stores to the copies
                         // below; one here would also wait for this thread's copies in flight (3 %
@@ -234,11 +252,11 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
             const uint32_t tS = tmem + kT_S, tD1 = tmem + kT_D1, tD4 = tmem + kT_D4;
             bool live = true;
             // the next unit's table entries are fetched while the current unit is processed
-            UnitInfo nxt = unit_info(p, ws, lay, min(cta, total_units - 1));
+            UnitInfo nxt = unit_info(p, ws, lay, min(cta, total_units - 1), done_tab);
             for (int unit = cta; unit < total_units && live; unit += n_ctas) {
                 const UnitInfo u = nxt;
-                nxt = unit_info(p, ws, lay, min(unit + n_ctas, total_units - 1));
-                if (u.skip) continue;
+                nxt = unit_info(p, ws, lay, min(unit + n_ctas, total_units - 1), done_tab);
+                if (u.skip || u.done) continue;
                 for (int j = 0; j < u.nc; ++j) {
                     const uint32_t g = gc + j;
                     const int st = g & 1;
@@ -326,13 +344,17 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
         // Every warp runs every group barrier and hand-over below, also after a wait has failed
         // (ok == false: later waits and all work are skipped), so that no warp is ever left alone
         // at a barrier.
-        UnitInfo nxt = unit_info(p, ws, lay, min(cta, total_units - 1));
+        UnitInfo nxt = unit_info(p, ws, lay, min(cta, total_units - 1), done_tab);
         for (int unit = cta; unit < total_units; unit += n_ctas) {
             const UnitInfo u = nxt;
-            nxt = unit_info(p, ws, lay, min(unit + n_ctas, total_units - 1));
+            nxt = unit_info(p, ws, lay, min(unit + n_ctas, total_units - 1), done_tab);
             const size_t tile_off = (static_cast<size_t>(u.bad_slot ? 0 : u.slot) * p.Hv + u.hv) * (kD * kD) +
                                     static_cast<size_t>(dv) * kD + half * 64;
+            if (u.done) continue;
             if (u.skip) {
+                if constexpr (kGated == 2) {
+                    if (tid == 0) done_w[unit] = 1;
+                }
                 if (u.bad_seq) continue;
                 if (u.bad_slot) {          // padding / out-of-range slot: zero rows, no state
                     if (u.slot >= p.num_slots && tid == 0) report(p.dev_status, kDevBadSlot);
@@ -427,6 +449,11 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
                         for (int j4 = 0; j4 < 64; j4 += 4)
                             *reinterpret_cast<float4*>(p.final_state + tile_off + j4) =
                                 make_float4(S[j4], S[j4 + 1], S[j4 + 2], S[j4 + 3]);
+                        // (every record of the unit has been loaded by now: no flag wait can
+                        // fail after this point, and any other failure is reported as an error)
+                        if constexpr (kGated == 2) {
+                            if (tid == 0) done_w[unit] = 1;
+                        }
                     }
                 }
                 if (!last) hand_over(&bar_s);
@@ -473,11 +500,11 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
             if (lane == 0) mbar_arrive(&bar_s);
         };
         bool preloaded = false;     // U~ of the chunk about to be processed is already in place
-        UnitInfo nxt = unit_info(p, ws, lay, min(cta, total_units - 1));
+        UnitInfo nxt = unit_info(p, ws, lay, min(cta, total_units - 1), done_tab);
         for (int unit = cta; unit < total_units; unit += n_ctas) {
             const UnitInfo u = nxt;
-            nxt = unit_info(p, ws, lay, min(unit + n_ctas, total_units - 1));
-            if (u.skip) continue;
+            nxt = unit_info(p, ws, lay, min(unit + n_ctas, total_units - 1), done_tab);
+            if (u.skip || u.done) continue;
             for (int j = 0; j < u.nc; ++j) {
                 const uint32_t g = gc + j;
                 const int buf = g & 1;
@@ -549,7 +576,7 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
     tc_fence_before_sync();
     __syncthreads();
     if (abort_flag != 0 && warp == kSIssueWarp && lane == 0) {
-        report(p.dev_status, kDevTimeout);
+        if (abort_flag == 1) report(p.dev_status, kDevTimeout);     // 2: a record not produced yet, no error
         // let copies already in flight land before the CTA's shared memory goes away
         mbar_wait(&bar_full[0], 0, 1u << 12);
         mbar_wait(&bar_full[1], 0, 1u << 12);

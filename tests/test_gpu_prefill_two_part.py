@@ -151,3 +151,32 @@ def test_two_part_production_replayed_from_a_cuda_graph():
     U.check_o(U.host_f64_from_bf16(o1), o_ref, U.O_REL_L2_PREFILL)
     U.check_state(f1.cpu().numpy().astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
 
+
+
+def test_serialised_launches_cost_time_not_results():
+    """split_permille = -2 launches the producers of the second part as an ordinary successor of
+    the state pass, which is what a tool that serialises launches would do: the state pass's waits
+    for their records run out (soon, and without an error), it marks what it finished, and the
+    last launch runs the other units once the records exist.  Same results, status clean."""
+    lens = [1500, 64, 0, 333, 700, 1]
+    p = I.prefill_inputs(lens, 2, 4, seed=78, init="normal")
+    num_slots = 8
+    slots = np.array([5, 0, 3, -1, 7, 2], np.int32)
+    init = np.zeros((num_slots, 4, 128, 128), np.float32)
+    for n in range(len(lens)):
+        if slots[n] >= 0:
+            init[slots[n]] = p["init_state"][n]
+    o_ref, S_ref, _ = oracle.prefill(p["q"], p["k"], p["v"], p["g"], p["beta"], p["cu_seqlens"],
+                                     init.astype(np.float64), slots, p["scale"], num_slots=num_slots)
+    o_par, S_par, st_par = run_prefill(p, "overlap", slot_idx=slots, num_slots=num_slots, init=init,
+                                       pool_fill=0.0, split_permille=-1)
+    for alias in (False, True):
+        kw = dict(alias=True) if alias else dict(pool_fill=0.0)
+        o, S, status = run_prefill(p, "overlap", slot_idx=slots, num_slots=num_slots, init=init.copy(),
+                                   split_permille=-2, **kw)
+        assert status == 0 and st_par == 0
+        assert np.array_equal(o, o_par)
+        keep = slots[slots >= 0]
+        assert np.array_equal(S[keep], S_par[keep])
+        U.check_o(o, o_ref, U.O_REL_L2_PREFILL)
+        U.check_state(S[keep].astype(np.float64), S_ref[keep], U.STATE_REL_L2_PREFILL)
