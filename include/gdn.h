@@ -202,6 +202,8 @@ int gdn_prefill(const void* q, const void* k, const void* v,
  * GDN_RECURRENT_MAX_SEQLEN tokens (by max_seqlen_hint if given, else by the
  * bound T) goes to the token-by-token kernel; anything longer to one of the
  * chunked variants (gdn_prefill_fused for a few long sequence-heads,
+ * gdn_prefill_overlap when max_seqlen_hint tells of chains of at least 40
+ * chunks and the sequence-heads number between a third and half of the SMs,
  * gdn_prefill_stream for chains longer than two chunks, more
  * sequence-heads than SMs or at most 16 sequences, else gdn_prefill_chunked).  Each route can also be called directly; arguments
  * are gdn_prefill's.  gdn_prefill_route answers which one gdn_prefill would take
@@ -215,6 +217,7 @@ int gdn_prefill(const void* q, const void* k, const void* v,
 #define GDN_ROUTE_CHUNKED   2
 #define GDN_ROUTE_FUSED     3
 #define GDN_ROUTE_STREAM    4
+#define GDN_ROUTE_OVERLAP   5
 int gdn_prefill_route(int32_t T, int32_t N, int32_t max_seqlen_hint, int32_t Hv,
                       int32_t sm_count, int32_t cooperative_launch);
 int gdn_prefill_chunked(const void* q, const void* k, const void* v,
@@ -284,9 +287,9 @@ int gdn_prefill_stream(const void* q, const void* k, const void* v,
  * time prevents).  If it does not happen the waits for records run out after
  * a fraction of a second, the state pass marks the (sequence, v-head) units it
  * has finished and the last launch runs the others once the records exist:
- * the results are the same, only time is lost.  For that reason gdn_prefill
- * never chooses this route by itself (it is not among gdn_prefill_route's
- * answers).  With CUDA_LAUNCH_BLOCKING set everything is produced first.
+ * the results are the same, only time is lost (so profile gdn_prefill_stream
+ * instead under such a tool).  With CUDA_LAUNCH_BLOCKING set everything is
+ * produced first.
  */
 int gdn_prefill_overlap(const void* q, const void* k, const void* v,
                         const float* g, const float* beta, const int32_t* cu_seqlens,

@@ -166,7 +166,7 @@ def gdn_state_transpose(state_pool, slot_idx=None, n=None, dev_status=None):
         raise GdnError(rc, "gdn_state_transpose")
 
 
-ROUTES = {0: "none", 1: "recurrent", 2: "chunked", 3: "fused", 4: "stream"}
+ROUTES = {0: "none", 1: "recurrent", 2: "chunked", 3: "fused", 4: "stream", 5: "overlap"}
 
 
 def gdn_prefill_route(T, N, max_seqlen_hint, Hv, sm_count=148, cooperative_launch=True) -> str:

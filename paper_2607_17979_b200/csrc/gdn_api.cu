@@ -252,11 +252,19 @@ int gdn_prefill_route(int32_t T, int32_t N, int32_t max_seqlen_hint, int32_t Hv,
     // Few (sequence, v-head) units and long sequences: the serial state pass would occupy only a
     // few SMs while the rest idle, so run it next to the record producers in one cooperative launch.
     if (cooperative_launch && units <= sm_count / 3 && longest > 16 * gdn::kChunk) return GDN_ROUTE_FUSED;
-    // gdn_prefill_overlap is never chosen here although it is the fastest route for long chains
-    // on at most half the SMs (10-15 % ahead of the three launches, 2-20 % ahead of the
-    // cooperative launch for several sequences): its state pass waits for a later launch, and
-    // that the two run at the same time is what the device does, not what CUDA promises.  The
-    // cooperative launch gives that promise; a caller who accepts the other asks for it by name.
+    // More units than the cooperative launch takes but at most half as many as SMs, with long
+    // chains (known only through the caller's hint): the state pass leaves half the machine free
+    // from the start, so part of the records is produced beside it (two sequences of 4096 tokens
+    // at 32 heads 261 -> 238 us, 4096 + 2048 230 -> 198 us, 8192 + 1024 382 -> 303 us; two chains of
+    // 32 chunks were 4 % slower, hence 40).  That route wants two launches to run side by side,
+    // which the device does but CUDA does not promise; if they do not, its last launch finishes
+    // the work (same results, about 0.1 s lost), so choosing it is safe.  Below a third of the
+    // SMs the cooperative launch is level with it or ahead; batches that fill the machine at
+    // first and free it as their short chains end would gain 5-12 %, but the records produced late
+    // are still dirty in L2 when the call ends and their write-back falls into whatever runs
+    // next, and batches of equal chains lose up to 7 %: those stay with the persistent pass.
+    if (max_seqlen_hint > 0 && units <= sm_count / 2 && longest >= 40 * gdn::kChunk)
+        return GDN_ROUTE_OVERLAP;
     // The persistent state pass has the shorter chunk step (its loader, issuer, chain and output
     // warps are separate) and does not pay a CTA start, a pipeline fill and a drain per unit:
     // measured faster whenever a chain is longer than two chunks or there are more units than
@@ -297,6 +305,7 @@ int gdn_prefill(const void* q, const void* k, const void* v, const float* g, con
     }
     const PrefillRoute route = route_id == GDN_ROUTE_FUSED     ? kRouteFused
                                : route_id == GDN_ROUTE_STREAM  ? kRouteStream
+                               : route_id == GDN_ROUTE_OVERLAP ? kRouteOverlap
                                                                : kRouteChunked;
     return prefill_chunked_impl(route, q, k, v, g, beta, cu_seqlens, init_state,
                                 final_state, slot_idx, o, T, N, Hqk, Hv, dk, dv, chunk, num_slots,

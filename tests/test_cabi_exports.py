@@ -120,9 +120,12 @@ def test_prefill_routing_rules_are_pure_host_arithmetic():
     assert r(1600, 16, 100, 4) == "stream" and r(1700, 17, 100, 4) == "chunked"
     assert r(8192, 128, 64, 32) == "stream" and r(296, 37, 8, 4) != "stream"        # 4096 / 148 units
     assert r(1184, 37, 32, 4) == "chunked" and r(1216, 38, 32, 4) == "stream"       # 148 / 152 units
-    # the two-part production (its state pass waits for a later launch) is never chosen
-    # automatically, whatever the hint
-    assert r(8192, 2, 4096, 32) == "stream" and r(8192, 2, 4096, 8) == "fused"
+    # the caller says how long the longest sequence is, chains of at least 40 chunks, more units
+    # than the cooperative launch takes and at most half as many as SMs: the two-part production
+    assert r(8192, 2, 4096, 32) == "overlap" and r(4000, 2, 3000, 32) == "overlap"
+    assert r(8192, 2, 0, 32) == "stream" and r(5118, 2, 2559, 32) == "stream"
+    assert r(8192, 2, 4096, 37) == "overlap" and r(8192, 2, 4096, 38) == "stream"   # 74 / 76 units
+    assert r(8192, 2, 4096, 24) == "fused" and r(8192, 2, 4096, 25) == "overlap"    # 48 / 50 units
     assert r(7680, 4, 4096, 32) == "stream" and r(6144, 3, 2048, 32) == "stream"
     # the thresholds follow the SM count given
     assert r(1184, 37, 32, 4, 100) == "stream"
