@@ -180,3 +180,31 @@ def test_serialised_launches_cost_time_not_results():
         assert np.array_equal(S[keep], S_par[keep])
         U.check_o(o, o_ref, U.O_REL_L2_PREFILL)
         U.check_state(S[keep].astype(np.float64), S_ref[keep], U.STATE_REL_L2_PREFILL)
+
+
+def test_host_buffer_prefill_behind_the_two_part_route():
+    """gdn_prefill_host on a batch that gdn_prefill sends to the two-part production: the copy of o
+    back to the host follows the last launch.  Five calls in a row, each compared bit for bit with
+    the device entry point."""
+    from paper_2607_17979_b200 import api
+    lens = [2700, 2600]
+    p = I.prefill_inputs(lens, 16, 32, seed=21, init="zero")
+    T, N = p["T"], p["N"]
+    assert api.gdn_prefill_route(T, N, max(lens), 32) == "overlap"
+    ws = torch.empty(api.gdn_prefill_workspace_bytes(T, N, 16, 32), dtype=torch.uint8, device="cuda")
+    o_dev, S_dev, st = run_prefill(p, "overlap", init=None)
+    assert st == 0
+    host = {n: U.dev_bf16(p[n]).cpu().pin_memory() for n in ("q", "k", "v")}
+    host.update({n: torch.from_numpy(p[n]).pin_memory() for n in ("g", "beta", "cu_seqlens")})
+    stage = torch.empty(api.gdn_prefill_host_staging_bytes(T, N, 16, 32), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for _ in range(5):
+        h_o = torch.zeros((T, 32, 128), dtype=torch.bfloat16).pin_memory()
+        final = torch.zeros((N, 32, 128, 128), dtype=torch.float32, device="cuda")
+        api.gdn_prefill_host(host["q"], host["k"], host["v"], host["g"], host["beta"],
+                             host["cu_seqlens"], None, final, None, h_o, p["scale"], stage, ws,
+                             max_seqlen_hint=max(lens), dev_status=status)
+        torch.cuda.synchronize()
+        assert np.array_equal(U.host_f64_from_bf16(h_o), o_dev)
+        assert np.array_equal(final.cpu().numpy(), S_dev)
+    assert int(status.item()) == 0
