@@ -285,7 +285,7 @@ int gdn_prefill_stream(const void* q, const void* k, const void* v,
  * at the same time, which programmatic dependent launch makes the device do
  * but which CUDA does not promise (and a tool that replays kernels one at a
  * time prevents).  If it does not happen the waits for records run out after
- * a fraction of a second, the state pass marks the (sequence, v-head) units it
+ * a few milliseconds, the state pass marks the (sequence, v-head) units it
  * has finished and the last launch runs the others once the records exist:
  * the results are the same, only time is lost (so profile gdn_prefill_stream
  * instead under such a tool).  With CUDA_LAUNCH_BLOCKING set everything is

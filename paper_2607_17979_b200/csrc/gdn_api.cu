@@ -258,7 +258,7 @@ int gdn_prefill_route(int32_t T, int32_t N, int32_t max_seqlen_hint, int32_t Hv,
     // at 32 heads 261 -> 238 us, 4096 + 2048 230 -> 198 us, 8192 + 1024 382 -> 303 us; two chains of
     // 32 chunks were 4 % slower, hence 40).  That route wants two launches to run side by side,
     // which the device does but CUDA does not promise; if they do not, its last launch finishes
-    // the work (same results, about 0.1 s lost), so choosing it is safe.  Below a third of the
+    // the work (same results, milliseconds lost), so choosing it is safe.  Below a third of the
     // SMs the cooperative launch is level with it or ahead; batches that fill the machine at
     // first and free it as their short chains end would gain 5-12 %, but the records produced late
     // are still dirty in L2 when the call ends and their write-back falls into whatever runs

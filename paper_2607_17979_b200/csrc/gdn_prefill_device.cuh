@@ -514,7 +514,7 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, vo
         if (mbar_try_wait(bar, parity)) return true;
         if ((i & 255u) == 255u && *abort_flag) return false;
     }
-    *abort_flag = 1;
+    if (*abort_flag == 0) *abort_flag = 1;      // keep an earlier, different reason
     return false;
 }
 

@@ -76,7 +76,9 @@ __device__ __forceinline__ UnitInfo unit_info(const PrefillParams& p, const uint
 }
 
 constexpr uint32_t kSpinFlagLimit = 1u << 22;
-constexpr uint32_t kSpinFlagLimitSoft = 1u << 17;
+// a few milliseconds: far longer than the producers ever lag when they do run beside the state
+// pass, far shorter than the other roles' mbarrier waits (which would report an error)
+constexpr uint32_t kSpinFlagLimitSoft = 1u << 13;
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
     uint32_t v;

@@ -153,15 +153,17 @@ def test_two_part_production_replayed_from_a_cuda_graph():
 
 
 
-def test_serialised_launches_cost_time_not_results():
+@pytest.mark.parametrize("lens,slots", [([1500, 64, 0, 333, 700, 1], [5, 0, 3, -1, 7, 2]),
+                                        ([1309, 1478, 993, 1452], [0, 1, 2, 3]),
+                                        ([1849, 67, 1043, 2012, 1319, 475, 1702], [7, 0, 5, 6, 4, 2, 3])])
+def test_serialised_launches_cost_time_not_results(lens, slots):
     """split_permille = -2 launches the producers of the second part as an ordinary successor of
     the state pass, which is what a tool that serialises launches would do: the state pass's waits
     for their records run out (soon, and without an error), it marks what it finished, and the
     last launch runs the other units once the records exist.  Same results, status clean."""
-    lens = [1500, 64, 0, 333, 700, 1]
     p = I.prefill_inputs(lens, 2, 4, seed=78, init="normal")
     num_slots = 8
-    slots = np.array([5, 0, 3, -1, 7, 2], np.int32)
+    slots = np.array(slots, np.int32)
     init = np.zeros((num_slots, 4, 128, 128), np.float32)
     for n in range(len(lens)):
         if slots[n] >= 0:
