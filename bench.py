@@ -9,6 +9,13 @@ leg's tokens/s and roofline are reported in the same JSON line under "prefill".
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
+Outside that timed step, rank 0 of a 1-GPU run also times the other three configurations and two
+measurement workloads, a few calls each, and adds them to the same JSON line: "decode_b1"
+(B=1 latency), "decode_paged" (B=256 of 512 slots, 1 GiB pool), "prefill_long" (one sequence of
+32768 tokens), "chain_bound" (the dependent chunk step of this run, from two single-sequence
+calls of 8192 and 16384 tokens) and "sweep" (mean latency over the short-prompt / small-batch
+shapes under CUDA-graph replay, with the host time per eager call).
+
 With N > 1 (launched by torch.distributed.run) every rank runs the same per-GPU workload on its
 own GPU (independent sequences, no data-path collective: weak scaling); the timed region is
 bracketed by a barrier and the per-step times are the max over ranks.
@@ -35,13 +42,22 @@ from paper_2607_17979_b200 import inputs as I  # noqa: E402
 DECODE_CFG, PREFILL_CFG = 1, 3
 DEC_POOLS, PRE_SETS = 8, 3
 TILE_BYTES = 128 * 128 * 4
+WORKLOAD = ("step = gdn_decode B=64 Hqk=16 Hv=32 d=128, 128 MiB fp32 state pool in place (configs[1]) "
+            "+ gdn_prefill 4 seqs {512,1024,2048,4096} = 7680 tokens, chunk 64 (configs[3])")
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures
-# (profiles/); None until a capture of that kernel exists.
-NCU_TRAFFIC_BYTES = {"decode": 213_381_376, "prefill": 730_488_832}
-# one dependent chunk step of the persistent state pass (clock stamps in a debug build: about 3630
-# cycles at 1965 MHz); the serial bound of a prefill call is the longest chain times this
-CHUNK_STEP_US = 1.85
+# single-sequence shapes whose time difference gives the dependent chunk step of this run
+CHAIN_SHORT, CHAIN_LONG = 8192, 16384
+EXTRA_REPS = 20          # timed calls of each workload outside the main step
+
+
+def ncu_traffic():
+    """dram__bytes_read.sum + dram__bytes_write.sum per call from the committed ncu captures:
+    profiles/traffic.json is rewritten whenever a summary under profiles/ is refreshed."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
+            return json.load(f)
+    except (OSError, ValueError):
+        return {}
 
 
 def peaks():
@@ -167,8 +183,7 @@ def run_reference(args):
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": 1e3 * float(np.mean(times)), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "decode B=64 Hqk=16 Hv=32 d=128 (configs[1]) + prefill 4 seqs, 7680 "
-                               "tokens (configs[3]), fp64 oracle on host cores", "l2": "host run"},
+        "config": {"workload": WORKLOAD, "l2": "host run: the fp64 oracle on the host cores"},
         "cpu_baseline": {"value": dec_gbs, "unit": "GB/s", "cores": last["cores"], "kind": "oracle",
                          "sample": last["sample"]},
         "prefill": {"metric": "gdn_prefill_tokens_per_s", "value": last["prefill_tok_s"],
@@ -289,57 +304,62 @@ def run_ours(args):
         sampler.start()
     dec_ms, pre_ms, spread = timed_region(step)
     e2e_dec_ms, e2e_pre_ms, _ = timed_region(e2e_step)
+    assert int(status.item()) == 0, "device status flagged during the benchmark"
+    extra = None
+    if rank == 0 and world == 1 and not args.no_extra:
+        # free the step's buffers first: the long-context workload alone needs 2 GB
+        del pools[1:], p_sets[1:], h_pre, h_po, stage_p, stage_d
+        torch.cuda.empty_cache()
+        extra = extra_workloads(api, torch, status, pre)
     clocks = sampler.stop() if rank == 0 else None
     assert int(status.item()) == 0, "device status flagged during the benchmark"
 
     if rank == 0:
         pk, pk_kind = peaks()
+        traffic = ncu_traffic()
         state_b, dec_b = decode_bytes(B, Hqk, Hv, False)
         pre_b, pre_f = prefill_bytes_flops(T, N, Hqk, Hv, False)
         dec_gbs = world * state_b / (dec_ms * 1e-3) / 1e9
         dec_ach = dec_b / (dec_ms * 1e-3) / 1e9
         pre_tok = world * T / (pre_ms * 1e-3)
-        pre_ach = pre_b / (pre_ms * 1e-3) / 1e9
-        pre_roof_ms = max(pre_b / (pk["hbm_gbs"] * 1e9),
-                          pre_f / (pk["bf16_tflops_sustained"] * 1e12)) * 1e3
         cpu = oracle_sample(dec, pre)
         h2d = sum(t.numel() * t.element_size() for t in h_dec.values())
-        h2d_p = sum(t.numel() * t.element_size() for t in h_pre.values()) + h_cu.numel() * 4
+        h2d_p = 2 * T * Hqk * 256 + T * Hv * 256 + 2 * T * Hv * 4 + (N + 1) * 4
+        pre_roof = prefill_roofline(pre_b, pre_f, pre_ms, pk, pk_kind, traffic.get("prefill_config3"))
+        dec_roof = {"kernel": "gdn decode (decode_kernel, one launch)", "bound": "hbm",
+                    "achieved": dec_ach, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                    "frac": dec_ach / pk["hbm_gbs"], "peak_kind": pk_kind,
+                    "frac_of_nominal_8TBps": dec_ach / 8000.0, "algorithmic_bytes": dec_b,
+                    "traffic": traffic.get("decode_config1")}
+        depth = -(-max(pre["seq_lens"]) // 64)
+        step_us = extra["chain_bound"]["chunk_step_us"] if extra else None
         line = {
             "metric": "gdn_decode_state_GBps", "value": dec_gbs, "unit": "GB/s",
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": dec_ms + pre_ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": "step = gdn_decode B=64 Hqk=16 Hv=32 d=128, 128 MiB fp32 state "
-                                   "pool in place (configs[1]) + gdn_prefill 4 seqs "
-                                   "{512,1024,2048,4096} = 7680 tokens, chunk 64 (configs[3])",
+            "config": {"workload": WORKLOAD,
                        "per_gpu": True,
                        "l2": f"inputs larger than L2: decode rotates over {DEC_POOLS} distinct 128 MiB "
                              f"state pools (1 GiB), prefill over {PRE_SETS} distinct input sets "
                              "(3 x 190 MB) plus its workspace",
                        "decode_ms": dec_ms, "prefill_ms": pre_ms,
                        "this_rank_spread": spread},
-            "roofline": {"kernel": "gdn decode", "bound": "hbm", "achieved": dec_ach,
-                         "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": dec_ach / pk["hbm_gbs"],
-                         "peak_kind": pk_kind, "frac_of_nominal_8TBps": dec_ach / 8000.0,
-                         "algorithmic_bytes": dec_b, "traffic": NCU_TRAFFIC_BYTES["decode"]},
+            # the dominant part of the step by time is the prefill call (all its launches)
+            "roofline": pre_roof,
+            "decode": {"metric": "gdn_decode_state_GBps", "value": dec_gbs, "unit": "GB/s",
+                       "ms": dec_ms, "roofline": dec_roof},
             "prefill": {"metric": "gdn_prefill_tokens_per_s", "value": pre_tok, "unit": "tokens/s",
                         "ms": pre_ms, "dtype": "bf16 operands, f32 accumulate and state",
-                        "roofline": {"kernel": "gdn prefill (all launches of one call)",
-                                     "bound": "hbm", "achieved": pre_ach, "peak": pk["hbm_gbs"],
-                                     "unit": "GB/s", "frac": pre_ach / pk["hbm_gbs"],
-                                     "peak_kind": pk_kind, "roofline_ms": pre_roof_ms,
-                                     "frac_of_roofline_time": pre_roof_ms / pre_ms,
-                                     "algorithmic_bytes": pre_b, "algorithmic_flops": pre_f,
-                                     "traffic": NCU_TRAFFIC_BYTES["prefill"]},
+                        "route": api.gdn_prefill_route(T, N, max(pre["seq_lens"]), Hv),
+                        "roofline": pre_roof,
                         # the serial part: the longest sequence's chunks, one dependent chunk step
-                        # each (step time from a cycle trace of the state pass, not from this run)
-                        "chain_bound": {"depth_chunks": -(-max(pre["seq_lens"]) // 64),
-                                        "chunk_step_us": CHUNK_STEP_US,
-                                        "ms": -(-max(pre["seq_lens"]) // 64) * CHUNK_STEP_US * 1e-3},
+                        # each, the step measured in this run (see "chain_bound")
+                        "chain_bound": {"depth_chunks": depth, "chunk_step_us": step_us,
+                                        "ms": None if step_us is None else depth * step_us * 1e-3},
                         "e2e": {"value": world * T / (e2e_pre_ms * 1e-3), "unit": "tokens/s",
                                 "h2d_bytes_per_step": h2d_p,
-                                "d2h_bytes_per_step": h_po.numel() * 2},
+                                "d2h_bytes_per_step": T * Hv * 256},
                         "cpu_baseline": {"value": cpu["prefill_tok_s"], "unit": "tokens/s"}},
             "cpu_baseline": {"value": cpu["decode_state_gbs"], "unit": "GB/s", "cores": cpu["cores"],
                              "kind": "oracle", "sample": cpu["sample"]},
@@ -351,8 +371,146 @@ def run_ours(args):
             "gpu_launches": args.steps * api.LAUNCHES_PER_STEP,
             "clocks": clocks,
         }
+        if extra:
+            for name in ("decode_b1", "decode_paged", "prefill_long", "chain_bound", "sweep"):
+                line[name] = extra[name]
+            for name, key in (("decode_paged", "decode_config2"), ("prefill_long", "prefill_config4")):
+                roof = line[name]["roofline"]
+                roof["peak"], roof["peak_kind"] = pk["hbm_gbs"], pk_kind
+                roof["frac"] = roof["achieved"] / pk["hbm_gbs"]
+                roof["traffic"] = traffic.get(key)
+            pl = line["prefill_long"]
+            roof_ms = max(pl["roofline"]["algorithmic_bytes"] / (pk["hbm_gbs"] * 1e9),
+                          pl["roofline"]["algorithmic_flops"] / (pk["bf16_tflops_sustained"] * 1e12)) * 1e3
+            pl["roofline"]["roofline_ms"] = roof_ms
+            pl["roofline"]["frac_of_roofline_time"] = roof_ms / pl["ms"]
+            pl["chain_bound"] = {"depth_chunks": 512, "chunk_step_us": step_us,
+                                 "ms": 512 * step_us * 1e-3}
         print(json.dumps(line))
     D.finish()
+
+
+def prefill_roofline(nbytes, flops, ms, pk, pk_kind, traffic):
+    roof_ms = max(nbytes / (pk["hbm_gbs"] * 1e9), flops / (pk["bf16_tflops_sustained"] * 1e12)) * 1e3
+    ach = nbytes / (ms * 1e-3) / 1e9
+    return {"kernel": "gdn prefill (all launches of one call)", "bound": "hbm", "achieved": ach,
+            "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": ach / pk["hbm_gbs"], "peak_kind": pk_kind,
+            "roofline_ms": roof_ms, "frac_of_roofline_time": roof_ms / ms,
+            "algorithmic_bytes": nbytes, "algorithmic_flops": flops, "traffic": traffic}
+
+
+def extra_workloads(api, torch, status, pre3):
+    """The configurations the main step does not time, plus the measured chunk step and the
+    small-shape sweep; EXTRA_REPS eager calls each, CUDA events, after 3 warm-up calls."""
+    import sweep as SW
+
+    def bf16(bits):
+        return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+    def dev(x):
+        return None if x is None else torch.from_numpy(x).cuda()
+
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def timed(fn, reps=EXTRA_REPS, flush=False):
+        for _ in range(3):
+            fn(0)
+        torch.cuda.synchronize()
+        ts = []
+        for i in range(reps):
+            if flush:
+                flush_buf.fill_(i & 255)        # 256 MB written: nothing of the workload stays in L2
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(i); e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        return float(np.mean(ts)), float(np.median(ts)), float(np.min(ts))
+
+    out = {}
+    # ---- configs[0]: decode B=1 (latency; about 1 MB moved, launch-bound: no fraction target)
+    d0 = I.make_config(0)
+    t0 = {n: (bf16(d0[n]) if n in "qkv" else dev(d0[n])) for n in ("q", "k", "v", "g", "beta")}
+    pool0 = dev(d0["state"])
+    o0 = torch.empty((1, d0["Hv"], 128), dtype=torch.bfloat16, device="cuda")
+    call0 = lambda i: api.gdn_decode(t0["q"], t0["k"], t0["v"], t0["g"], t0["beta"], pool0, None, o0,
+                                     d0["scale"], status)
+    cold = timed(call0, flush=True)
+    hot = timed(call0)
+    graph_us = SW._time(lambda: call0(0), 200)
+    _, b0 = decode_bytes(1, d0["Hqk"], d0["Hv"], False)
+    out["decode_b1"] = {"workload": "configs[0]: gdn_decode B=1 Hqk=4 Hv=8", "unit": "us",
+                        "value": cold[1] * 1e3, "us_cold_l2_median": cold[1] * 1e3,
+                        "us_hot_l2_median": hot[1] * 1e3, "us_graph_replay": graph_us,
+                        "algorithmic_bytes": b0,
+                        "note": "eager CUDA-event times of one tiny launch include the launch itself; "
+                                "graph replay is device time per call, L2-resident"}
+    del pool0
+
+    # ---- configs[2]: decode B=256 of 512 slots, rotating over 2 pools of 1 GiB
+    d2 = I.make_config(2)
+    t2 = {n: (bf16(d2[n]) if n in "qkv" else dev(d2[n])) for n in ("q", "k", "v", "g", "beta")}
+    idx2 = dev(d2["slot_idx"])
+    pools2 = [dev(d2["state"]) for _ in range(2)]
+    o2 = torch.empty((256, 32, 128), dtype=torch.bfloat16, device="cuda")
+    call2 = lambda i: api.gdn_decode(t2["q"], t2["k"], t2["v"], t2["g"], t2["beta"], pools2[i & 1],
+                                     idx2, o2, d2["scale"], status)
+    m2 = timed(call2)
+    sb2, b2 = decode_bytes(256, 16, 32, True)
+    out["decode_paged"] = {"workload": "configs[2]: gdn_decode B=256 of 512 slots, 1 GiB fp32 pool, "
+                                       "int32 slot indices, 2 pools in rotation",
+                           "metric": "gdn_decode_state_GBps", "unit": "GB/s",
+                           "value": sb2 / (m2[0] * 1e-3) / 1e9, "ms": m2[0], "ms_median": m2[1],
+                           "roofline": {"kernel": "gdn decode (decode_kernel, one launch)",
+                                        "bound": "hbm", "achieved": b2 / (m2[0] * 1e-3) / 1e9,
+                                        "unit": "GB/s", "algorithmic_bytes": b2,
+                                        "frac_of_nominal_8TBps": b2 / (m2[0] * 1e-3) / 1e9 / 8000.0}}
+    del pools2, d2, t2
+
+    # ---- a prefill call on given lengths (16 / 32 heads), mean ms
+    def prefill_ms(p, reps):
+        T, N, Hv = p["T"], p["N"], p["Hv"]
+        t = {n: (bf16(p[n]) if n in "qkv" else dev(p[n])) for n in ("q", "k", "v", "g", "beta")}
+        cu, init = dev(p["cu_seqlens"]), dev(p["init_state"])
+        final = torch.empty((N, Hv, 128, 128), dtype=torch.float32, device="cuda")
+        o = torch.empty((T, Hv, 128), dtype=torch.bfloat16, device="cuda")
+        ws = torch.empty(api.gdn_prefill_workspace_bytes(T, N, p["Hqk"], Hv), dtype=torch.uint8,
+                         device="cuda")
+        hint = max(p["seq_lens"])
+        return timed(lambda i: api.gdn_prefill(t["q"], t["k"], t["v"], t["g"], t["beta"], cu, init,
+                                               final, None, o, p["scale"], ws, max_seqlen_hint=hint,
+                                               dev_status=status), reps)
+
+    # ---- configs[4]: one sequence of 32768 tokens (inputs 0.8 GB + workspace: larger than L2)
+    p4 = I.make_config(4)
+    m4 = prefill_ms(p4, max(5, EXTRA_REPS // 2))
+    b4, f4 = prefill_bytes_flops(p4["T"], 1, 16, 32, True)
+    out["prefill_long"] = {"workload": "configs[4]: gdn_prefill 1 sequence of 32768 tokens, Hqk=16 "
+                                       "Hv=32, alpha in [0.95,1), fp32 initial state",
+                           "metric": "gdn_prefill_tokens_per_s", "unit": "tokens/s",
+                           "value": p4["T"] / (m4[0] * 1e-3), "ms": m4[0], "ms_median": m4[1],
+                           "route": api.gdn_prefill_route(p4["T"], 1, p4["T"], 32),
+                           "roofline": {"kernel": "gdn prefill (all launches of one call)",
+                                        "bound": "hbm", "achieved": b4 / (m4[0] * 1e-3) / 1e9,
+                                        "unit": "GB/s", "algorithmic_bytes": b4,
+                                        "algorithmic_flops": f4}}
+    del p4
+    torch.cuda.empty_cache()
+
+    # ---- the dependent chunk step: two single sequences whose lengths differ by 128 chunks
+    ms_s = prefill_ms(I.prefill_inputs([CHAIN_SHORT], 16, 32, seed=I.BASE_SEED + 1), EXTRA_REPS)
+    ms_l = prefill_ms(I.prefill_inputs([CHAIN_LONG], 16, 32, seed=I.BASE_SEED + 2), EXTRA_REPS)
+    dchunks = (CHAIN_LONG - CHAIN_SHORT) // 64
+    out["chain_bound"] = {"chunk_step_us": (ms_l[1] - ms_s[1]) * 1e3 / dchunks,
+                          "how": f"(median ms of 1 x {CHAIN_LONG} tokens - median ms of 1 x "
+                                 f"{CHAIN_SHORT} tokens) / {dchunks} chunks, Hv=32, this run",
+                          "ms_short": ms_s[1], "ms_long": ms_l[1],
+                          "route": api.gdn_prefill_route(CHAIN_LONG, 1, CHAIN_LONG, 32)}
+    torch.cuda.empty_cache()
+
+    # ---- small-shape sweep (CUDA-graph replay) and host time per eager call (C++ loop)
+    _, summary = SW.run(reps=100, multi=False)
+    out["sweep"] = summary
+    return out
 
 
 def main():
@@ -361,6 +519,8 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extra", action="store_true",
+                    help="time the main step only (skip the other configurations and the sweep)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

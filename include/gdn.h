@@ -22,7 +22,10 @@
  * Common rules for every call below
  *   - Every pointer is DEVICE memory owned by the caller unless a comment says
  *     "host".  The library allocates nothing and keeps no state between calls
- *     except where an entry point's own comment says otherwise.
+ *     except where an entry point's own comment says otherwise (and except a few
+ *     facts about each device, looked up on first use and remembered: its SM
+ *     count, whether it launches cooperatively, which kernels had their shared
+ *     memory limit raised).
  *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*) and return
  *     without synchronising.  No device data is read on the host.
  *   - Return value: 0 = enqueued; negative = rejected before any launch and
@@ -330,8 +333,9 @@ int gdn_prefill_recurrent(const void* q, const void* k, const void* v,
  * workspace_bytes; inputs and outputs are still the caller's buffers.
  *   - A batch needing more scratch than the array holds
  *     (gdn_prefill_workspace_bytes(...) > GDN_STATIC_WORKSPACE_BYTES) returns
- *     GDN_ERR_LIMIT and nothing is launched.  With Hv = 32 the array covers up to
- *     18 chunks of 64 tokens (floor(T/64) + N <= 18), e.g. 1024 tokens in 2 sequences.
+ *     GDN_ERR_LIMIT and nothing is launched.  The scratch is 74 240 bytes per
+ *     chunk slot and v-head plus small tables, so with Hv = 32 the array covers
+ *     14 chunk slots (floor(T/64) + N <= 14), e.g. 768 tokens in 2 sequences.
  *   - The call itself allocates and frees nothing.  The first call on each
  *     device looks up the array's device address (one cudaGetSymbolAddress, with
  *     that device current) and caches it; make that first call outside of any
@@ -381,6 +385,32 @@ int gdn_prefill_host(const void* q, const void* k, const void* v,
                      void* staging, size_t staging_bytes,
                      void* workspace, size_t workspace_bytes,
                      int32_t* dev_status, void* stream);
+
+/*
+ * gdn_host_us_per_decode_call / gdn_host_us_per_prefill_call - measurement aids
+ * (no counterpart in the paper, whose remark they serve: small-batch decode is
+ * dominated by launch overhead and dispatch).  Each makes one untimed call, then
+ * `reps` back-to-back calls of gdn_decode / gdn_prefill with the given arguments
+ * on `stream`, and returns the mean HOST time per call in microseconds (argument
+ * checks, tensor-map encoding and kernel launches; the stream is synchronised
+ * before and after, outside the clock).  A negative return is the GDN_ERR_* code
+ * of a rejected call.  The calls really run: the state pool / outputs are
+ * updated reps + 1 times.  dev_status is not used.
+ */
+double gdn_host_us_per_decode_call(const void* q, const void* k, const void* v,
+                                   const float* g, const float* beta,
+                                   float* state_pool, const int32_t* slot_idx, void* o,
+                                   int32_t B, int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv,
+                                   int32_t num_slots, float scale, void* stream, int32_t reps);
+double gdn_host_us_per_prefill_call(const void* q, const void* k, const void* v,
+                                    const float* g, const float* beta, const int32_t* cu_seqlens,
+                                    const float* init_state, float* final_state,
+                                    const int32_t* slot_idx, void* o,
+                                    int32_t T, int32_t N, int32_t max_seqlen_hint,
+                                    int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv, int32_t chunk,
+                                    int32_t num_slots, float scale,
+                                    void* workspace, size_t workspace_bytes,
+                                    void* stream, int32_t reps);
 
 /* Human-readable name of a return code (static storage, never NULL). */
 const char* gdn_status_string(int code);

@@ -20,7 +20,8 @@ EXPORTS = ("gdn_decode", "gdn_prefill_workspace_bytes", "gdn_prefill", "gdn_pref
            "gdn_state_transpose", "gdn_decode_host", "gdn_decode_host_staging_bytes",
            "gdn_prefill_host", "gdn_prefill_host_staging_bytes",
            "gdn_prefill_recurrent",
-           "gdn_prefill_static", "gdn_prefill_static_workspace_bytes", "gdn_status_string",
+           "gdn_prefill_static", "gdn_prefill_static_workspace_bytes",
+           "gdn_host_us_per_decode_call", "gdn_host_us_per_prefill_call", "gdn_status_string",
            "gdn_last_cuda_error_string", "gdn_version")
 
 # kernels one call enqueues (for the benchmark's launch count)
@@ -71,6 +72,10 @@ _lib.gdn_prefill_host_staging_bytes.restype = _Z
 _lib.gdn_prefill_host_staging_bytes.argtypes = [_I] * 4
 _lib.gdn_prefill_host.restype = ctypes.c_int
 _lib.gdn_prefill_host.argtypes = [_P] * 10 + [_I] * 9 + [_F, _P, _Z, _P, _Z, _P, _P]
+_lib.gdn_host_us_per_decode_call.restype = ctypes.c_double
+_lib.gdn_host_us_per_decode_call.argtypes = [_P] * 8 + [_I] * 6 + [_F, _P, _I]
+_lib.gdn_host_us_per_prefill_call.restype = ctypes.c_double
+_lib.gdn_host_us_per_prefill_call.argtypes = [_P] * 10 + [_I] * 9 + [_F, _P, _Z, _P, _I]
 _lib.gdn_status_string.restype = ctypes.c_char_p
 _lib.gdn_status_string.argtypes = [ctypes.c_int]
 _lib.gdn_last_cuda_error_string.restype = ctypes.c_char_p
@@ -227,6 +232,10 @@ def gdn_prefill_recurrent(q, k, v, g, beta, cu_seqlens, init_state, final_state,
         raise GdnError(rc, "gdn_prefill_recurrent")
 
 
+# chunk slots (floor(T/64) + N) the built-in array of gdn_prefill_static covers at 32 v-heads
+STATIC_MAX_CHUNK_SLOTS_HV32 = 14
+
+
 def gdn_prefill_static_workspace_bytes() -> int:
     """Size of the scratch array built into the library (the limit gdn_prefill_static enforces)."""
     return int(_lib.gdn_prefill_static_workspace_bytes())
@@ -251,6 +260,42 @@ def gdn_prefill_static(q, k, v, g, beta, cu_seqlens, init_state, final_state, sl
         float(scale), _dev(dev_status, torch.int32, "dev_status", True), _stream())
     if rc != 0:
         raise GdnError(rc, "gdn_prefill_static")
+
+
+def gdn_host_us_per_decode_call(q, k, v, g, beta, state_pool, slot_idx, o, scale, reps=100) -> float:
+    """Mean host microseconds inside one gdn_decode call (a C++ loop of ``reps`` calls; see gdn.h)."""
+    B, Hqk, dk = q.shape
+    _, Hv, dv = v.shape
+    us = _lib.gdn_host_us_per_decode_call(
+        _dev(q, torch.bfloat16, "q"), _dev(k, torch.bfloat16, "k"), _dev(v, torch.bfloat16, "v"),
+        _dev(g, torch.float32, "g"), _dev(beta, torch.float32, "beta"),
+        _dev(state_pool, torch.float32, "state_pool"),
+        _dev(slot_idx, torch.int32, "slot_idx", True), _dev(o, torch.bfloat16, "o"),
+        B, Hqk, Hv, dk, dv, state_pool.shape[0], float(scale), _stream(), int(reps))
+    if us < 0:
+        raise GdnError(int(us), "gdn_host_us_per_decode_call")
+    return float(us)
+
+
+def gdn_host_us_per_prefill_call(q, k, v, g, beta, cu_seqlens, init_state, final_state, slot_idx, o,
+                                 scale, workspace, max_seqlen_hint=0, chunk=64, reps=50) -> float:
+    """Mean host microseconds inside one gdn_prefill call (a C++ loop of ``reps`` calls)."""
+    T, Hqk, dk = q.shape
+    _, Hv, dv = v.shape
+    N = cu_seqlens.shape[0] - 1
+    us = _lib.gdn_host_us_per_prefill_call(
+        _dev(q, torch.bfloat16, "q"), _dev(k, torch.bfloat16, "k"), _dev(v, torch.bfloat16, "v"),
+        _dev(g, torch.float32, "g"), _dev(beta, torch.float32, "beta"),
+        _dev(cu_seqlens, torch.int32, "cu_seqlens"),
+        _dev(init_state, torch.float32, "init_state", True),
+        _dev(final_state, torch.float32, "final_state"),
+        _dev(slot_idx, torch.int32, "slot_idx", True), _dev(o, torch.bfloat16, "o"),
+        T, N, int(max_seqlen_hint), Hqk, Hv, dk, dv, int(chunk), final_state.shape[0],
+        float(scale), _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(),
+        int(reps))
+    if us < 0:
+        raise GdnError(int(us), "gdn_host_us_per_prefill_call")
+    return float(us)
 
 
 def _host(t, dtype, name, allow_none=False):

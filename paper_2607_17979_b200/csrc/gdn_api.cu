@@ -281,10 +281,11 @@ int gdn_prefill(const void* q, const void* k, const void* v, const float* g, con
                 int32_t Hqk, int32_t Hv, int32_t dk, int32_t dv, int32_t chunk,
                 int32_t num_slots, float scale, void* workspace, size_t workspace_bytes,
                 int32_t* dev_status, void* stream) {
-    int dev = 0, sms = 148, coop = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess) {
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+    int sms = 148, coop = 0;
+    gdn::DeviceInfo di;
+    if (gdn::device_info(&di) == cudaSuccess) {
+        sms = di.sms;
+        coop = di.cooperative;
     }
     const int route_id = gdn_prefill_route(T, N, max_seqlen_hint, Hv, sms, coop);
     if (chunk == gdn::kChunk && route_id == GDN_ROUTE_RECURRENT) {

@@ -52,6 +52,17 @@ struct PrefillParams {
     int32_t* dev_status;
 };
 
+// The current device's SM count and cooperative-launch support, queried once per device.
+struct DeviceInfo {
+    int device, sms, cooperative;
+};
+cudaError_t device_info(DeviceInfo* out);
+// Raises a kernel's dynamic shared memory limit on the current device, once per device.
+cudaError_t ensure_dynamic_smem(const void* kernel, int bytes);
+template <class K> inline cudaError_t ensure_dynamic_smem(K* kernel, int bytes) {
+    return ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), bytes);
+}
+
 cudaError_t launch_decode(const DecodeParams& p, cudaStream_t stream);
 cudaError_t launch_decode_multi(const DecodeMultiParams& mp, cudaStream_t stream);
 cudaError_t launch_gate(const __nv_bfloat16* a, const __nv_bfloat16* b, const float* A_log,

@@ -112,9 +112,8 @@ cudaError_t launch_decode(const DecodeParams& p, cudaStream_t stream) {
     if (units == 0) return cudaSuccess;
     // below about two CTAs per SM of whole tiles, quarter tiles spread the same bytes over four
     // times as many SMs (the state rows are independent)
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess)
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    DeviceInfo di;
+    const int sms = device_info(&di) == cudaSuccess ? di.sms : 148;
     if (units < 2LL * sms)
         decode_kernel<1><<<static_cast<unsigned>(units * 4), kDecodeThreads, 0, stream>>>(p);
     else   // half tiles at three CTAs per SM: measured 0.5-1 % faster than whole tiles at two

@@ -294,9 +294,8 @@ decode_multi_kv_kernel(const DecodeMultiParams mp) {
 cudaError_t launch_decode_multi(const DecodeMultiParams& mp, cudaStream_t stream) {
     const long long units = static_cast<long long>(mp.d.B) * mp.d.Hv;
     if (units == 0) return cudaSuccess;
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess)
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    DeviceInfo di;
+    const int sms = device_info(&di) == cudaSuccess ? di.sms : 148;
     // fewer than two whole tiles per SM: quarter tiles spread the bytes over more SMs
     const bool split = units < 2LL * sms;
     const unsigned grid = static_cast<unsigned>(split ? units * 4 : units);

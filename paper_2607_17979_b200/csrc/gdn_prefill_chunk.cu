@@ -546,7 +546,7 @@ bool prefill_tables_inline(const ChunkedParams& cp) {
 cudaError_t launch_prefill_intra(const TensorMaps& maps, const ChunkedParams& cp, cudaStream_t stream,
                                  bool inline_tables) {
     auto kernel = inline_tables ? prefill_intra_kernel<true> : prefill_intra_kernel<false>;
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kIntraSmem);
+    cudaError_t e = ensure_dynamic_smem(kernel, kIntraSmem);
     if (e != cudaSuccess) return e;
     dim3 grid(cp.lay.max_chunks, cp.p.Hv);
     return launch_dependent(kernel, grid, dim3(kIntraThreads), kIntraSmem, stream, maps, cp.p, cp.ws,
@@ -555,8 +555,7 @@ cudaError_t launch_prefill_intra(const TensorMaps& maps, const ChunkedParams& cp
 
 cudaError_t launch_prefill_chunked(const ChunkedParams& cp, cudaStream_t stream) {
     const PrefillParams& p = cp.p;
-    cudaError_t e = cudaFuncSetAttribute(prefill_state_kernel,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, kStateSmem);
+    cudaError_t e = ensure_dynamic_smem(prefill_state_kernel, kStateSmem);
     if (e != cudaSuccess) return e;
     TensorMaps maps;
     if (!make_prefill_tensor_maps(&maps, p)) return cudaErrorInvalidValue;

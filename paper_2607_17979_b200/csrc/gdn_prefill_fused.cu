@@ -315,14 +315,12 @@ cudaError_t launch_prefill_ranked_prep(const ChunkedParams& cp, cudaStream_t str
 
 cudaError_t launch_prefill_fused(const ChunkedParams& cp, cudaStream_t stream) {
     const PrefillParams& p = cp.p;
-    int dev = 0, sms = 0, coop = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+    DeviceInfo di;
+    cudaError_t e = device_info(&di);
     if (e != cudaSuccess) return e;
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+    const int sms = di.sms, coop = di.cooperative;
     if (!coop || sms < 2) return cudaErrorNotSupported;
-    e = cudaFuncSetAttribute(prefill_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kFusedSmem);
+    e = ensure_dynamic_smem(prefill_fused_kernel, kFusedSmem);
     if (e != cudaSuccess) return e;
     TensorMaps maps;
     if (!make_prefill_tensor_maps(&maps, p)) return cudaErrorInvalidValue;

@@ -188,21 +188,17 @@ prefill_state_stream_rest_kernel(const __grid_constant__ TensorMaps maps, const 
 
 cudaError_t launch_prefill_overlap(const ChunkedParams& cp, cudaStream_t stream, int split_permille) {
     const PrefillParams& p = cp.p;
-    int dev = 0, sms = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+    DeviceInfo di;
+    cudaError_t e = device_info(&di);
     if (e != cudaSuccess) return e;
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    e = cudaFuncSetAttribute(prefill_state_stream_gated_kernel,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmem);
+    const int sms = di.sms;
+    e = ensure_dynamic_smem(prefill_state_stream_gated_kernel, kStreamSmem);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(prefill_state_stream_rest_kernel,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmem);
+    e = ensure_dynamic_smem(prefill_state_stream_rest_kernel, kStreamSmem);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(prefill_intra_first_kernel,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, kIntraSmem);
+    e = ensure_dynamic_smem(prefill_intra_first_kernel, kIntraSmem);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(prefill_intra_second_kernel,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, kIntraSmem);
+    e = ensure_dynamic_smem(prefill_intra_second_kernel, kIntraSmem);
     if (e != cudaSuccess) return e;
     TensorMaps maps;
     if (!make_prefill_tensor_maps(&maps, p)) return cudaErrorInvalidValue;

@@ -29,12 +29,11 @@ prefill_state_stream_kernel(const __grid_constant__ TensorMaps maps, const Prefi
 // kernel over all items; then this kernel on min(units, SMs) CTAs.
 cudaError_t launch_prefill_stream(const ChunkedParams& cp, cudaStream_t stream) {
     const PrefillParams& p = cp.p;
-    int dev = 0, sms = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+    DeviceInfo di;
+    cudaError_t e = device_info(&di);
     if (e != cudaSuccess) return e;
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    e = cudaFuncSetAttribute(prefill_state_stream_kernel,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmem);
+    const int sms = di.sms;
+    e = ensure_dynamic_smem(prefill_state_stream_kernel, kStreamSmem);
     if (e != cudaSuccess) return e;
     TensorMaps maps;
     if (!make_prefill_tensor_maps(&maps, p)) return cudaErrorInvalidValue;

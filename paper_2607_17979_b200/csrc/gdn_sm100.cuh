@@ -1,6 +1,6 @@
 // Thin inline-PTX wrappers for the sm_100a machinery the prefill kernels use:
 // mbarriers with bounded waits, TMA (tiled tensor loads and linear bulk copies,
-// never multicast), tensor memory allocation, tcgen05.mma / commit / ld / st
+// plain per-CTA copies only), tensor memory allocation, tcgen05.mma / commit / ld / st
 // and the shared-memory and instruction descriptors.
 #pragma once
 #include <cuda_runtime.h>

@@ -402,3 +402,28 @@ def test_bad_cu_seqlens_rejected():
         oracle.prefill(p["qb"], p["kb"], p["vb"], p["g"], p["beta"], np.array([0, 3, 2, 4], np.int32))
     with pytest.raises(ValueError):
         oracle.prefill(p["qb"], p["kb"], p["vb"], p["g"], p["beta"], np.array([0, 3], np.int32))
+
+
+def test_thread_count_never_changes_a_bit():
+    """Threads only split the independent (sequence, v-head) units among themselves: one thread,
+    three threads and the default count must give identical bits for prefill and for decode."""
+    rs = np.random.default_rng(19)
+    lens = [9, 0, 14, 3, 21]
+    T = sum(lens); Hqk, Hv, dk, dv = 2, 6, 8, 5
+    p = rand_problem(rs, T, Hqk, Hv, dk, dv)
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    S0 = rs.standard_normal((5, Hv, dv, dk))
+    runs = [oracle.prefill(p["qb"], p["kb"], p["vb"], p["g"], p["beta"], cu, S0.copy(), scale=0.7,
+                           n_threads=n) for n in (1, 3, 0)]
+    for o, S, _ in runs[1:]:
+        assert np.array_equal(o, runs[0][0]) and np.array_equal(S, runs[0][1])
+    B = 7
+    d = rand_problem(rs, B, Hqk, Hv, dk, dv)
+    pool0 = rs.standard_normal((B, Hv, dv, dk))
+    outs = []
+    for n in (1, 3, 0):
+        pool = pool0.copy()
+        o, _ = oracle.decode(d["qb"], d["kb"], d["vb"], d["g"], d["beta"], pool, None, 0.7, n_threads=n)
+        outs.append((o, pool))
+    for o, pool in outs[1:]:
+        assert np.array_equal(o, outs[0][0]) and np.array_equal(pool, outs[0][1])

@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2607_17979_b200 import inputs as I
 import gpu_util as U
 
@@ -48,6 +49,40 @@ def test_static_workspace_entry_point_matches_gdn_prefill_on_two_calls_in_a_row(
         assert np.abs(o_s - o_r).max() <= U.O_MAX_ABS and U.rel_l2(o_s, o_r) <= U.O_REL_L2_PREFILL
         assert U.rel_l2(S_s.astype(np.float64), S_r.astype(np.float64)) <= U.STATE_REL_L2_PREFILL
         assert np.array_equal(o_s, o_r) and np.array_equal(S_s, S_r)
+        # and against the fp64 oracle, like every other entry point
+        o_ref, S_ref, _ = oracle.prefill(p["q"], p["k"], p["v"], p["g"], p["beta"], p["cu_seqlens"],
+                                         None if p["init_state"] is None
+                                         else p["init_state"].astype(np.float64), None, p["scale"])
+        U.check_o(o_s, o_ref, U.O_REL_L2_PREFILL)
+        U.check_state(S_s.astype(np.float64), S_ref, U.STATE_REL_L2_PREFILL)
+
+
+def test_static_workspace_entry_point_at_the_edge_of_its_array():
+    """With 32 v-heads and two sequences: the largest batch whose scratch still fits the array runs
+    and reproduces gdn_prefill; one more chunk is refused with GDN_ERR_LIMIT and writes nothing."""
+    from paper_2607_17979_b200 import api
+    limit = api.gdn_prefill_static_workspace_bytes()
+    chunks = 1
+    while api.gdn_prefill_workspace_bytes(64 * (chunks + 1), 2, 16, 32) <= limit:
+        chunks += 1
+    T_fit = 64 * chunks                       # floor(T/64) + N = chunks + 2 chunk slots
+    assert api.gdn_prefill_workspace_bytes(T_fit, 2, 16, 32) <= limit
+    assert api.gdn_prefill_workspace_bytes(T_fit + 64, 2, 16, 32) > limit
+    assert chunks + 2 == api.STATIC_MAX_CHUNK_SLOTS_HV32      # the figure the header states
+    fit = I.prefill_inputs([T_fit - 100, 100], 16, 32, seed=4103, init="normal")
+    o_s, S_s = _run(fit, static=True)
+    o_r, S_r = _run(fit, static=False)
+    assert np.array_equal(o_s, o_r) and np.array_equal(S_s, S_r)
+    over = I.prefill_inputs([T_fit - 100 + 64, 100], 16, 32, seed=4104, init="zero")
+    final = torch.zeros((2, 32, 128, 128), dtype=torch.float32, device="cuda")
+    o = torch.zeros((over["T"], 32, 128), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(api.GdnError) as e:
+        api.gdn_prefill_static(U.dev_bf16(over["q"]), U.dev_bf16(over["k"]), U.dev_bf16(over["v"]),
+                               U.dev(over["g"]), U.dev(over["beta"]), U.dev(over["cu_seqlens"]), None,
+                               final, None, o, over["scale"])
+    assert e.value.code == -7
+    torch.cuda.synchronize()
+    assert float(final.abs().max()) == 0 and float(o.float().abs().max()) == 0
 
 
 def test_static_workspace_entry_point_rejects_batches_beyond_its_array():
