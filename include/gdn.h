@@ -59,8 +59,8 @@ extern "C" {
 
 /*
  * gdn_decode - one token of the gated delta rule for each of B sequences
- * (paper: "Decode receives a prior state and computes ... new recurrent
- * updates"; here exactly one update per sequence per call).
+ * (paper, subsection "Gated Delta Net", the decode regime: a prior state plus a
+ * few new updates; here exactly one update per sequence per call).
  *
  * For entry i and v-head hv, with slot = slot_idx ? slot_idx[i] : i and the
  * tile S = state_pool[slot][hv]:
@@ -88,9 +88,9 @@ int gdn_decode(const void* q, const void* k, const void* v,
 /*
  * gdn_decode_multi - L >= 1 new tokens of the gated delta rule for each of B
  * sequences in one call, applied in order, with a choice of state orientation
- * (paper, same subsection: decode "computes a small number of new recurrent
- * updates"; the paper's decode routes differ in "state layout", one of them
- * working on the transposed tile).  The result equals L successive gdn_decode
+ * (paper, same subsection: the decode regime applies a few new updates to a
+ * prior state, and the paper's decode routes differ in how the state tile is
+ * laid out, one of them working on the transposed tile).  The result equals L successive gdn_decode
  * calls; the state tile is read and written once for all L tokens.
  *
  *   q, k        bf16 [B][L][Hqk][dk]
@@ -162,9 +162,9 @@ size_t gdn_prefill_workspace_bytes(int32_t T, int32_t N, int32_t Hqk, int32_t Hv
 
 /*
  * gdn_prefill - the same recurrence over N packed variable-length sequences
- * (paper: "Prefill evaluates a whole sequence and returns both outputs and the
- * final state ... parallelizing the recurrence through chunked matrix
- * operations while applying the log-domain gate consistently").  The result is
+ * (paper, subsection "Gated Delta Net", the prefill regime: whole sequences in,
+ * outputs and final state out, the recurrence evaluated chunk by chunk as
+ * matrix products with the gate kept in the log domain).  The result is
  * the token-by-token recurrence's; chunking only re-associates it.
  *
  * Sequence n owns tokens cu_seqlens[n] .. cu_seqlens[n+1]-1 and the state tile
@@ -266,9 +266,9 @@ int gdn_prefill_stream(const void* q, const void* k, const void* v,
                        int32_t* dev_status, void* stream);
 
 /*
- * gdn_prefill_overlap - the chunked algorithm (same section of the paper as
- * gdn_prefill: the prefill regime of the gated delta rule, "through chunked
- * matrix operations") with the intra-chunk work cut in two around the
+ * gdn_prefill_overlap - the chunked algorithm (same subsection of the paper as
+ * gdn_prefill: the prefill regime of the gated delta rule) with the
+ * intra-chunk work cut in two around the
  * persistent state pass: the records the chains need first are produced
  * before the state pass starts, the others beside it, on the SMs that hold no
  * live chain, each published through a flag the state pass waits for (bounded

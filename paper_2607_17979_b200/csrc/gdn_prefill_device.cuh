@@ -9,7 +9,7 @@ namespace gdn {
 using namespace sm100;
 
 constexpr int kIntraThreads = 256;
-constexpr uint32_t kIntraTmemCols = 128;
+constexpr uint32_t kIntraTmemCols = 128;    // the Gram accumulator, then W^T in the same columns; U~^T
 constexpr int kLdA = 68;               // row stride (floats) of the fp32 A / T matrix
 // Shared memory map (bytes from a 1024-aligned base).  Regions are reused as their contents die
 // so that four CTAs fit on an SM:
@@ -49,13 +49,18 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
-// One 16x8 output tile  C += A[16 x 8*ksteps] * B[8*ksteps x 8]  on mma.sync m16n8k8 with both
-// operands split into tf32 hi + lo parts (three products; the lo*lo term is dropped), which keeps
-// fp32-level accuracy.  A, B: fp32 row-major in shared memory; g = lane / 4, t = lane % 4.
-__device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo) {
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(hi) : "f"(x));
-    const float rem = x - __uint_as_float(hi);
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(lo) : "f"(rem));
+// One 16x8 output tile  C += A[16 x 8*ksteps] * B[8*ksteps x 8]  on mma.sync m16n8k8 with tf32
+// operands (rounded to nearest, one product per k-step) and fp32 accumulation.  A, B: fp32
+// row-major in shared memory; g = lane / 4, t = lane % 4.
+// Accuracy: these products only form the OFF-diagonal blocks of T = (I + A)^-1 from blocks that
+// are exact to fp32; an operand error of 2^-11 there moves the final state by about 1e-5 of its
+// norm on random keys and 3e-4 when all keys coincide (the worst case for the solve), against
+// 1.6e-4 and 1.4e-3 from the bf16 operands of the other products.  Split operands (three
+// products per k-step) bought nothing measurable and cost 2.3x the instructions.
+__device__ __forceinline__ uint32_t to_tf32(float x) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return r;
 }
 __device__ __forceinline__ void mma_m16n8k8_tf32(float (&c)[4], const uint32_t (&a)[4],
                                                  const uint32_t (&b)[2]) {
@@ -65,108 +70,23 @@ __device__ __forceinline__ void mma_m16n8k8_tf32(float (&c)[4], const uint32_t (
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
 }
-__device__ __forceinline__ void mma_tile_tf32x3(const float* A, int lda, const float* B, int ldb,
-                                                int ksteps, float (&c)[4], int g, int t) {
-    float c1[4] = {0.f, 0.f, 0.f, 0.f}, c2[4] = {0.f, 0.f, 0.f, 0.f};   // separate dependency chains
-#pragma unroll 4
-    for (int ks = 0; ks < ksteps; ++ks) {
+template <int kSteps>
+__device__ __forceinline__ void mma_tile_tf32(const float* A, int lda, const float* B, int ldb,
+                                              float (&c)[4], int g, int t) {
+    uint32_t a[kSteps][4], b[kSteps][2];
+#pragma unroll
+    for (int ks = 0; ks < kSteps; ++ks) {          // every load first, then the products
         const float* a_ = A + 8 * ks;
         const float* b_ = B + (8 * ks) * ldb;
-        const float af[4] = {a_[g * lda + t], a_[(g + 8) * lda + t], a_[g * lda + t + 4],
-                             a_[(g + 8) * lda + t + 4]};
-        const float bf[2] = {b_[t * ldb + g], b_[(t + 4) * ldb + g]};
-        uint32_t ah[4], al[4], bh[2], bl[2];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) split_tf32(af[i], ah[i], al[i]);
-#pragma unroll
-        for (int i = 0; i < 2; ++i) split_tf32(bf[i], bh[i], bl[i]);
-        mma_m16n8k8_tf32(c1, al, bh);
-        mma_m16n8k8_tf32(c2, ah, bl);
-        mma_m16n8k8_tf32(c, ah, bh);
+        a[ks][0] = to_tf32(a_[g * lda + t]);
+        a[ks][1] = to_tf32(a_[(g + 8) * lda + t]);
+        a[ks][2] = to_tf32(a_[g * lda + t + 4]);
+        a[ks][3] = to_tf32(a_[(g + 8) * lda + t + 4]);
+        b[ks][0] = to_tf32(b_[t * ldb + g]);
+        b[ks][1] = to_tf32(b_[(t + 4) * ldb + g]);
     }
 #pragma unroll
-    for (int i = 0; i < 4; ++i) c[i] += c1[i] + c2[i];
-}
-
-// T = (I + A)^{-1} for the strictly lower-triangular 64x64 A in sA (row-major, stride kLdA),
-// in place, by 256 threads: four 16x16 diagonal blocks by forward substitution in fp32, then the
-// off-diagonal blocks by block elimination at block sizes 16 and 32
-//     [[Ta, 0], [X, Tb]],  X = -Tb (A_ba Ta),
-// whose small products run on the legacy mma.sync path with split-tf32 operands (fp32-level
-// accuracy; tcgen05 needs M >= 64).  Rows past the chunk's length `len` are zero in A, so the
-// elimination levels that only touch such rows are skipped.  Ends with a group barrier.
-template <class Sync>
-__device__ __forceinline__ void solve_unit_lower_64(float* sA, float* scr, int tid, Sync sync,
-                                                    const int len = 64) {
-    // ---- diagonal blocks: thread (I, j) computes column j of (I + A_II)^{-1}, right-looking
-    if (tid < 64) {
-        const int I = tid >> 4, j = tid & 15;
-        float* blk = sA + (16 * I) * kLdA + 16 * I;
-        float t[16];
-#pragma unroll
-        for (int r = 0; r < 16; ++r) t[r] = (r == j) ? 1.f : 0.f;
-#pragma unroll
-        for (int i = 0; i < 15; ++i) {
-            const float ti = t[i];
-#pragma unroll
-            for (int r = i + 1; r < 16; ++r) t[r] = fmaf(-blk[r * kLdA + i], ti, t[r]);
-        }
-        __syncwarp();                      // every column of the block has read A_II
-#pragma unroll
-        for (int r = 0; r < 16; ++r) blk[r * kLdA + j] = t[r];
-    }
-    // the scratch borrows shared memory whose previous contents thread 0 is still bulk-storing
-    if (tid == 0) bulk_wait_read_all();
-    sync();
-    if (len <= 16) return;                 // every off-diagonal block lies in zero rows
-    // ---- off-diagonal blocks on the tensor cores (mma.sync m16n8k8, 3xTF32: fp32-level accuracy)
-    const int warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-    // 16-blocks (1,0) and (3,2): X = A_IJ T_JJ, then T_IJ = -T_II X.  Four 16x8 tiles, warps 0-3.
-    {
-        const int pr = warp >> 1, nb = warp & 1;            // pair, 8-column block
-        const int I = 2 * pr + 1, J = 2 * pr;
-        float* X = scr + pr * (16 * 24);
-        float c[4] = {0.f, 0.f, 0.f, 0.f};
-        if (warp < 4) {
-            mma_tile_tf32x3(sA + (16 * I) * kLdA + 16 * J, kLdA, sA + (16 * J) * kLdA + 16 * J + 8 * nb,
-                            kLdA, 2, c, g, t);
-            *reinterpret_cast<float2*>(X + g * 24 + 8 * nb + 2 * t) = make_float2(c[0], c[1]);
-            *reinterpret_cast<float2*>(X + (g + 8) * 24 + 8 * nb + 2 * t) = make_float2(c[2], c[3]);
-        }
-        sync();
-        if (warp < 4) {
-            c[0] = c[1] = c[2] = c[3] = 0.f;
-            mma_tile_tf32x3(sA + (16 * I) * kLdA + 16 * I, kLdA, X + 8 * nb, 24, 2, c, g, t);
-            float* dst = sA + (16 * I) * kLdA + 16 * J + 8 * nb;
-            *reinterpret_cast<float2*>(dst + g * kLdA + 2 * t) = make_float2(-c[0], -c[1]);
-            *reinterpret_cast<float2*>(dst + (g + 8) * kLdA + 2 * t) = make_float2(-c[2], -c[3]);
-        }
-    }
-    sync();
-    if (len <= 32) return;                 // block (1,0) of the 32-level lies in zero rows
-    // 32-block (1,0): Y = A_ba Ta, then X = -Tb Y.  Eight 16x8 tiles, one per warp.
-    {
-        const int mr = warp >> 2, nb = warp & 3;
-        float c[4] = {0.f, 0.f, 0.f, 0.f};
-        mma_tile_tf32x3(sA + (32 + 16 * mr) * kLdA, kLdA, sA + 8 * nb, kLdA, 4, c, g, t);
-        *reinterpret_cast<float2*>(scr + (16 * mr + g) * 40 + 8 * nb + 2 * t) = make_float2(c[0], c[1]);
-        *reinterpret_cast<float2*>(scr + (16 * mr + g + 8) * 40 + 8 * nb + 2 * t) = make_float2(c[2], c[3]);
-        sync();
-        c[0] = c[1] = c[2] = c[3] = 0.f;
-        mma_tile_tf32x3(sA + (32 + 16 * mr) * kLdA + 32, kLdA, scr + 8 * nb, 40, 4, c, g, t);
-        float* dst = sA + (32 + 16 * mr) * kLdA + 8 * nb;
-        *reinterpret_cast<float2*>(dst + g * kLdA + 2 * t) = make_float2(-c[0], -c[1]);
-        *reinterpret_cast<float2*>(dst + (g + 8) * kLdA + 2 * t) = make_float2(-c[2], -c[3]);
-    }
-    sync();
-}
-
-// Lane 0 polls the mbarrier (bounded), the other lanes block at the warp barrier instead of
-// competing for issue slots; returns the same verdict on every lane.
-__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity) {
-    int ok = 1;
-    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity) ? 1 : 0;
-    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+    for (int ks = 0; ks < kSteps; ++ks) mma_m16n8k8_tf32(c, a[ks], b[ks]);
 }
 
 __device__ __forceinline__ uint32_t scale_bf16x2(uint32_t packed, float f) {
@@ -183,6 +103,85 @@ struct IntraStatics {
     alignas(16) float s_bg[kChunk];    // beta_r e^{b_r}
     alignas(16) float s_eb[kChunk];    // e^{b_r}
 };
+
+// Diagonal 16x16 blocks of T = (I + A)^{-1} by forward substitution in fp32, in place in sA
+// (row-major, stride kLdA); run by warps 0 and 1: thread (I, j) computes column j of
+// (I + A_II)^{-1}, right-looking.
+__device__ __forceinline__ void solve_diagonal_blocks(float* sA, int tid) {
+    const int I = tid >> 4, j = tid & 15;
+    float* blk = sA + (16 * I) * kLdA + 16 * I;
+    float t[16];
+#pragma unroll
+    for (int r = 0; r < 16; ++r) t[r] = (r == j) ? 1.f : 0.f;
+#pragma unroll
+    for (int i = 0; i < 15; ++i) {
+        const float ti = t[i];
+#pragma unroll
+        for (int r = i + 1; r < 16; ++r) t[r] = fmaf(-blk[r * kLdA + i], ti, t[r]);
+    }
+    __syncwarp();                      // every column of the block has read A_II
+#pragma unroll
+    for (int r = 0; r < 16; ++r) blk[r * kLdA + j] = t[r];
+}
+
+// The off-diagonal blocks of T, given its diagonal 16x16 blocks, by block elimination at block
+// sizes 16 and 32
+//     [[Ta, 0], [X, Tb]],  X = -Tb (A_ba Ta),
+// whose small products run on the legacy mma.sync path (tcgen05 needs M >= 64).  Rows past the
+// chunk's length `len` are zero in A, so the elimination levels that only touch such rows are
+// skipped.  256 threads; ends with a group barrier.
+template <class Sync>
+__device__ __forceinline__ void solve_merge_levels(float* sA, float* scr, int tid, Sync sync,
+                                                   const int len) {
+    if (len <= 16) return;                 // every off-diagonal block lies in zero rows
+    const int warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+    // 16-blocks (1,0) and (3,2): X = A_IJ T_JJ, then T_IJ = -T_II X.  Four 16x8 tiles, warps 0-3.
+    {
+        const int pr = warp >> 1, nb = warp & 1;            // pair, 8-column block
+        const int I = 2 * pr + 1, J = 2 * pr;
+        float* X = scr + pr * (16 * 24);
+        float c[4] = {0.f, 0.f, 0.f, 0.f};
+        if (warp < 4) {
+            mma_tile_tf32<2>(sA + (16 * I) * kLdA + 16 * J, kLdA, sA + (16 * J) * kLdA + 16 * J + 8 * nb,
+                             kLdA, c, g, t);
+            *reinterpret_cast<float2*>(X + g * 24 + 8 * nb + 2 * t) = make_float2(c[0], c[1]);
+            *reinterpret_cast<float2*>(X + (g + 8) * 24 + 8 * nb + 2 * t) = make_float2(c[2], c[3]);
+        }
+        sync();
+        if (warp < 4) {
+            c[0] = c[1] = c[2] = c[3] = 0.f;
+            mma_tile_tf32<2>(sA + (16 * I) * kLdA + 16 * I, kLdA, X + 8 * nb, 24, c, g, t);
+            float* dst = sA + (16 * I) * kLdA + 16 * J + 8 * nb;
+            *reinterpret_cast<float2*>(dst + g * kLdA + 2 * t) = make_float2(-c[0], -c[1]);
+            *reinterpret_cast<float2*>(dst + (g + 8) * kLdA + 2 * t) = make_float2(-c[2], -c[3]);
+        }
+    }
+    sync();
+    if (len <= 32) return;                 // block (1,0) of the 32-level lies in zero rows
+    // 32-block (1,0): Y = A_ba Ta, then X = -Tb Y.  Eight 16x8 tiles, one per warp.
+    {
+        const int mr = warp >> 2, nb = warp & 3;
+        float c[4] = {0.f, 0.f, 0.f, 0.f};
+        mma_tile_tf32<4>(sA + (32 + 16 * mr) * kLdA, kLdA, sA + 8 * nb, kLdA, c, g, t);
+        *reinterpret_cast<float2*>(scr + (16 * mr + g) * 40 + 8 * nb + 2 * t) = make_float2(c[0], c[1]);
+        *reinterpret_cast<float2*>(scr + (16 * mr + g + 8) * 40 + 8 * nb + 2 * t) = make_float2(c[2], c[3]);
+        sync();
+        c[0] = c[1] = c[2] = c[3] = 0.f;
+        mma_tile_tf32<4>(sA + (32 + 16 * mr) * kLdA + 32, kLdA, scr + 8 * nb, 40, c, g, t);
+        float* dst = sA + (32 + 16 * mr) * kLdA + 8 * nb;
+        *reinterpret_cast<float2*>(dst + g * kLdA + 2 * t) = make_float2(-c[0], -c[1]);
+        *reinterpret_cast<float2*>(dst + (g + 8) * kLdA + 2 * t) = make_float2(-c[2], -c[3]);
+    }
+    sync();
+}
+
+// Lane 0 polls the mbarrier (bounded), the other lanes block at the warp barrier instead of
+// competing for issue slots; returns the same verdict on every lane.
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity) {
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity) ? 1 : 0;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
 
 // The intra-chunk quantities of one (chunk, v-head) item, computed by a group of 256 threads
 // (tid = 0..255 within the group; its warps must be CTA warps 0-3 mod 4 aligned, because a warp
@@ -301,20 +300,27 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
 #pragma unroll
         for (int step = 0; step < 2; ++step) {
             const int cbase = colhalf * 32 + step * 16;
-            uint32_t x[16];
-            tmem_ld16(tG + lane_base + cbase, x);
-            tmem_wait_ld();
             float val[16];
+            // a 16-column block that lies wholly above the diagonal for every row of the warp is
+            // zero (warp-uniform test: no accumulator read, no exponentials)
+            if (cbase > (row & 32) + 31) {
 #pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) {
-                const float4 bb = *reinterpret_cast<const float4*>(st.s_b2 + cbase + 4 * q4);
-                const float bv[4] = {bb.x, bb.y, bb.z, bb.w};
+                for (int jj = 0; jj < 16; ++jj) val[jj] = 0.f;
+            } else {
+                uint32_t x[16];
+                tmem_ld16(tG + lane_base + cbase, x);
+                tmem_wait_ld();
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int jj = 4 * q4 + e;
-                    const bool keep = cbase + jj <= limit;
-                    const float dec = ex2_approx(keep ? br2 - bv[e] : 0.f);   // e^{b_r - b_i}
-                    val[jj] = keep ? rowscale * dec * __uint_as_float(x[jj]) : 0.f;
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    const float4 bb = *reinterpret_cast<const float4*>(st.s_b2 + cbase + 4 * q4);
+                    const float bv[4] = {bb.x, bb.y, bb.z, bb.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int jj = 4 * q4 + e;
+                        const bool keep = cbase + jj <= limit;
+                        const float dec = ex2_approx(keep ? br2 - bv[e] : 0.f);   // e^{b_r - b_i}
+                        val[jj] = keep ? rowscale * dec * __uint_as_float(x[jj]) : 0.f;
+                    }
                 }
             }
             if (is_p) {
@@ -335,10 +341,16 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
             }
         }
     }
-    {   // Q rows scaled by scale * e^{b_r}, in place (the Gram product has consumed Q): this is the Qg image
-#pragma unroll
-        for (int it = 0; it < 4; ++it) {
-            const int idx = tid + it * kIntraThreads;          // 1024 16-byte pieces
+    tc_fence_before_sync();
+    sync();
+    // Two jobs side by side: warps 0-1 invert the four diagonal 16x16 blocks of I + A (a serial
+    // forward substitution per column, 64 threads' worth of work), warps 2-7 scale the Q rows by
+    // scale * e^{b_r} in place (the Gram product has consumed Q): that is the Qg image.
+    if (warp < 2) {
+        solve_diagonal_blocks(sA, tid);
+    } else {
+#pragma unroll 2
+        for (int idx = tid - 64; idx < 1024; idx += kIntraThreads - 64) {      // 1024 16-byte pieces
             const int halfq = idx >> 9, rem = idx & 511;
             const int r = rem >> 3;
             uint4* ptr = reinterpret_cast<uint4*>(smem + kI_QK + halfq * 16384 + rem * 16);
@@ -348,18 +360,20 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
             w.z = scale_bf16x2(w.z, f); w.w = scale_bf16x2(w.w, f);
             *ptr = w;
         }
+        fence_proxy_async_smem();
     }
-    fence_proxy_async_smem();
-    tc_fence_before_sync();
     sync();
     if (tid == 0) {
-        // Qg is final: store it now; its shared memory is reused from the solve on
+        // Qg is final: store it now; its shared memory is reused by the solve's merge levels.
+        // The scratch of those levels borrows the first Q half, which this bulk store is still
+        // reading: wait for the reads (not for the writes to land) before anyone goes on.
         bulk_store(rec + kRecQg, smem + kI_QK, 8192);
         bulk_store(rec + kRecQg + 8192, smem + kI_QK + 16384, 8192);
         bulk_commit();
+        bulk_wait_read_all();
     }
-
-    solve_unit_lower_64(sA, reinterpret_cast<float*>(smem + kI_Scr), tid, sync, ci.len);
+    sync();
+    solve_merge_levels(sA, reinterpret_cast<float*>(smem + kI_Scr), tid, sync, ci.len);
 
     uint32_t tu_lo[2][4];    // T diag(beta) - bf16(T diag(beta)), parked until T_w is dead
     {   // T (fp32, row-major) -> bf16 B operands T diag(beta e^b), T diag(beta) (hi, lo)
@@ -495,15 +509,11 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
     return true;
 }
 
-constexpr int kStateEpiWarps = 8;
-constexpr int kStateEpiThreads = kStateEpiWarps * 32;
-constexpr int kStateThreads = kStateEpiThreads + 32;
 constexpr uint32_t kStateTmemCols = 512;
 constexpr uint32_t kS_Rec = 0;                 // record image (74240 B, padded to 74752)
 constexpr uint32_t kS_K = 74752;               // K tile, 2 halves [64 x 128 B]
 constexpr uint32_t kStageBytes = 74752 + 16384;                 // 91136
 constexpr uint32_t kS_Out = 2 * kStageBytes;   // o staging [64 tokens][128 dv] bf16
-constexpr uint32_t kStateSmem = 2 * kStageBytes + 16384 + 1024;
 // TMEM columns
 constexpr uint32_t kT_D1 = 0, kT_Y = 64 /* two tiles of 64 */, kT_D4 = 192, kT_S = 320, kT_U = 384,
                    kT_Us = 416, kT_UsLo = 448;
@@ -523,10 +533,6 @@ __device__ __forceinline__ bool warp_wait_or_abort(uint64_t* bar, uint32_t parit
     int ok = 1;
     if ((threadIdx.x & 31) == 0) ok = wait_or_abort(bar, parity, abort_flag) ? 1 : 0;
     return __shfl_sync(0xffffffffu, ok, 0) != 0;
-}
-
-__device__ __forceinline__ void epi_group_sync() {      // the 256 epilogue threads only
-    asm volatile("bar.sync 1, %0;" ::"n"(kStateEpiThreads) : "memory");
 }
 
 
