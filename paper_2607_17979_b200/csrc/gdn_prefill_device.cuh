@@ -13,7 +13,7 @@ constexpr uint32_t kIntraTmemCols = 128;    // the Gram accumulator, then W^T in
 constexpr int kLdA = 68;               // row stride (floats) of the fp32 A / T matrix
 // Shared memory map (bytes from a 1024-aligned base).  Regions are reused as their contents die
 // so that four CTAs fit on an SM:
-//   R1  Q/K tiles.  Q half 0 -> Qg image (stored early) -> solve scratch -> T_w -> T_u(lo);
+//   R1  Q/K tiles.  Q half 0 -> Qg image (stored early) -> T_w -> T_u(lo);
 //       Q half 1 -> Qg image -> T_u(hi);  K halves -> W image.
 //   R2  A, then T, in fp32 -> V tile (loaded after the solve).
 // The P image goes straight from registers to the record; T_u(lo) waits in registers until the
@@ -21,13 +21,11 @@ constexpr int kLdA = 68;               // row stride (floats) of the fp32 A / T 
 constexpr uint32_t kI_QK = 0;          // 2 halves x [128 rows x 128 B]: rows 0-63 Q, 64-127 K
 constexpr uint32_t kI_Tw = 0;          // over Q half 0: T diag(beta e^b) [64 r x 64 i] bf16, K-major
 constexpr uint32_t kI_TuLo = 0;        // ... and later the bf16 remainder of T diag(beta)
-constexpr uint32_t kI_Scr = 0;         // ... and, between the two, the solve scratch, fp32 [32][40]
 constexpr uint32_t kI_Tu = 16384;      // over Q half 1: T diag(beta) rounded to bf16
 constexpr uint32_t kI_A = 32768;       // A, then T in place: fp32 [64][kLdA]
 constexpr uint32_t kI_V = 32768;       // over A: 2 halves x [64 x 128 B]
 constexpr uint32_t kI_End = kI_A + 64 * kLdA * 4;      // 50176
 constexpr uint32_t kIntraSmem = kI_End + 1024;         // + alignment slack
-static_assert(32 * 40 * 4 <= 8192, "solve scratch must fit in the Q half it borrows");
 static_assert(kI_End % 1024 == 0 && 64 * kLdA * 4 >= 16384, "V tile must fit over A");
 
 struct TensorMaps {
@@ -104,75 +102,97 @@ struct IntraStatics {
     alignas(16) float s_eb[kChunk];    // e^{b_r}
 };
 
-// Diagonal 16x16 blocks of T = (I + A)^{-1} by forward substitution in fp32, in place in sA
-// (row-major, stride kLdA); run by warps 0 and 1: thread (I, j) computes column j of
-// (I + A_II)^{-1}, right-looking.
-__device__ __forceinline__ void solve_diagonal_blocks(float* sA, int tid) {
-    const int I = tid >> 4, j = tid & 15;
-    float* blk = sA + (16 * I) * kLdA + 16 * I;
-    float t[16];
+// T = (I + A)^{-1} for the strictly lower-triangular 64x64 A in sA (fp32, row-major, stride kLdA),
+// in place, in two warp-local stages that need no barrier wider than a warp:
+//   solve_blocks_16_32: a warp inverts two neighbouring diagonal 16x16 blocks by forward
+//     substitution (thread (I, j) computes column j of (I + A_II)^{-1}, right-looking) and joins
+//     them into the inverse of their 32x32 block,
+//   solve_merge_64: a warp computes an 8-column block of the last off-diagonal 32x32 block,
+// both by block elimination  [[Ta, 0], [X, Tb]],  X = -Tb (A_ba Ta),  whose small products run on
+// the legacy mma.sync path (tcgen05 needs M >= 64).  The intermediate product A_ba Ta changes
+// from accumulator to operand layout through the block of sA that mirrors X above the diagonal
+// (zero in A and in T), which the warp clears again.
+// Warp `pr` (0 or 1) of the group: diagonal blocks 2 pr, 2 pr + 1 and block (2 pr + 1, 2 pr).
+__device__ __forceinline__ void solve_blocks_16_32(float* sA, const int pr, const int lane,
+                                                   const int len) {
+    {
+        const int I = 2 * pr + (lane >> 4), j = lane & 15;
+        float* blk = sA + (16 * I) * kLdA + 16 * I;
+        float t[16];
 #pragma unroll
-    for (int r = 0; r < 16; ++r) t[r] = (r == j) ? 1.f : 0.f;
+        for (int r = 0; r < 16; ++r) t[r] = (r == j) ? 1.f : 0.f;
 #pragma unroll
-    for (int i = 0; i < 15; ++i) {
-        const float ti = t[i];
+        for (int i = 0; i < 15; ++i) {
+            const float ti = t[i];
 #pragma unroll
-        for (int r = i + 1; r < 16; ++r) t[r] = fmaf(-blk[r * kLdA + i], ti, t[r]);
+            for (int r = i + 1; r < 16; ++r) t[r] = fmaf(-blk[r * kLdA + i], ti, t[r]);
+        }
+        __syncwarp();                      // every column of the block has read A_II
+#pragma unroll
+        for (int r = 0; r < 16; ++r) blk[r * kLdA + j] = t[r];
     }
-    __syncwarp();                      // every column of the block has read A_II
+    if (len <= 32 * pr + 16) return;       // block (2 pr + 1, 2 pr) lies in rows past the chunk's length: zero
+    __syncwarp();
+    const int g = lane >> 2, t = lane & 3;
+    const int I = 2 * pr + 1, J = 2 * pr;
+    float* A_IJ = sA + (16 * I) * kLdA + 16 * J;
+    float* X = sA + (16 * J) * kLdA + 16 * I;          // the mirror block, zero on entry
 #pragma unroll
-    for (int r = 0; r < 16; ++r) blk[r * kLdA + j] = t[r];
+    for (int nb = 0; nb < 2; ++nb) {                   // X = A_IJ T_JJ
+        float c[4] = {0.f, 0.f, 0.f, 0.f};
+        mma_tile_tf32<2>(A_IJ, kLdA, sA + (16 * J) * kLdA + 16 * J + 8 * nb, kLdA, c, g, t);
+        *reinterpret_cast<float2*>(X + g * kLdA + 8 * nb + 2 * t) = make_float2(c[0], c[1]);
+        *reinterpret_cast<float2*>(X + (g + 8) * kLdA + 8 * nb + 2 * t) = make_float2(c[2], c[3]);
+    }
+    __syncwarp();
+    float c[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+    for (int nb = 0; nb < 2; ++nb)                     // T_IJ = -T_II X
+        mma_tile_tf32<2>(sA + (16 * I) * kLdA + 16 * I, kLdA, X + 8 * nb, kLdA, c[nb], g, t);
+    __syncwarp();                                      // every lane has read X and A_IJ
+    {
+        const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+        float* xr = X + (lane >> 1) * kLdA + 8 * (lane & 1);
+        *reinterpret_cast<float4*>(xr) = zero;
+        *reinterpret_cast<float4*>(xr + 4) = zero;
+    }
+#pragma unroll
+    for (int nb = 0; nb < 2; ++nb) {
+        float* dst = A_IJ + 8 * nb;
+        *reinterpret_cast<float2*>(dst + g * kLdA + 2 * t) = make_float2(-c[nb][0], -c[nb][1]);
+        *reinterpret_cast<float2*>(dst + (g + 8) * kLdA + 2 * t) = make_float2(-c[nb][2], -c[nb][3]);
+    }
 }
 
-// The off-diagonal blocks of T, given its diagonal 16x16 blocks, by block elimination at block
-// sizes 16 and 32
-//     [[Ta, 0], [X, Tb]],  X = -Tb (A_ba Ta),
-// whose small products run on the legacy mma.sync path (tcgen05 needs M >= 64).  Rows past the
-// chunk's length `len` are zero in A, so the elimination levels that only touch such rows are
-// skipped.  256 threads; ends with a group barrier.
-template <class Sync>
-__device__ __forceinline__ void solve_merge_levels(float* sA, float* scr, int tid, Sync sync,
-                                                   const int len) {
-    if (len <= 16) return;                 // every off-diagonal block lies in zero rows
-    const int warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-    // 16-blocks (1,0) and (3,2): X = A_IJ T_JJ, then T_IJ = -T_II X.  Four 16x8 tiles, warps 0-3.
-    {
-        const int pr = warp >> 1, nb = warp & 1;            // pair, 8-column block
-        const int I = 2 * pr + 1, J = 2 * pr;
-        float* X = scr + pr * (16 * 24);
-        float c[4] = {0.f, 0.f, 0.f, 0.f};
-        if (warp < 4) {
-            mma_tile_tf32<2>(sA + (16 * I) * kLdA + 16 * J, kLdA, sA + (16 * J) * kLdA + 16 * J + 8 * nb,
-                             kLdA, c, g, t);
-            *reinterpret_cast<float2*>(X + g * 24 + 8 * nb + 2 * t) = make_float2(c[0], c[1]);
-            *reinterpret_cast<float2*>(X + (g + 8) * 24 + 8 * nb + 2 * t) = make_float2(c[2], c[3]);
-        }
-        sync();
-        if (warp < 4) {
-            c[0] = c[1] = c[2] = c[3] = 0.f;
-            mma_tile_tf32<2>(sA + (16 * I) * kLdA + 16 * I, kLdA, X + 8 * nb, 24, c, g, t);
-            float* dst = sA + (16 * I) * kLdA + 16 * J + 8 * nb;
-            *reinterpret_cast<float2*>(dst + g * kLdA + 2 * t) = make_float2(-c[0], -c[1]);
-            *reinterpret_cast<float2*>(dst + (g + 8) * kLdA + 2 * t) = make_float2(-c[2], -c[3]);
-        }
-    }
-    sync();
-    if (len <= 32) return;                 // block (1,0) of the 32-level lies in zero rows
-    // 32-block (1,0): Y = A_ba Ta, then X = -Tb Y.  Eight 16x8 tiles, one per warp.
-    {
-        const int mr = warp >> 2, nb = warp & 3;
+// Columns 8 nb .. 8 nb + 7 (nb = 0..3) of the 32x32 block (1, 0), by one warp, given the inverses
+// of the two diagonal 32x32 blocks.
+__device__ __forceinline__ void solve_merge_64(float* sA, const int nb, const int lane) {
+    const int g = lane >> 2, t = lane & 3;
+    float* Y = sA + 32 + 8 * nb;                       // rows 0-31 of the mirror block, zero on entry
+#pragma unroll
+    for (int mr = 0; mr < 2; ++mr) {                   // Y = A_ba Ta
         float c[4] = {0.f, 0.f, 0.f, 0.f};
         mma_tile_tf32<4>(sA + (32 + 16 * mr) * kLdA, kLdA, sA + 8 * nb, kLdA, c, g, t);
-        *reinterpret_cast<float2*>(scr + (16 * mr + g) * 40 + 8 * nb + 2 * t) = make_float2(c[0], c[1]);
-        *reinterpret_cast<float2*>(scr + (16 * mr + g + 8) * 40 + 8 * nb + 2 * t) = make_float2(c[2], c[3]);
-        sync();
-        c[0] = c[1] = c[2] = c[3] = 0.f;
-        mma_tile_tf32<4>(sA + (32 + 16 * mr) * kLdA + 32, kLdA, scr + 8 * nb, 40, c, g, t);
-        float* dst = sA + (32 + 16 * mr) * kLdA + 8 * nb;
-        *reinterpret_cast<float2*>(dst + g * kLdA + 2 * t) = make_float2(-c[0], -c[1]);
-        *reinterpret_cast<float2*>(dst + (g + 8) * kLdA + 2 * t) = make_float2(-c[2], -c[3]);
+        *reinterpret_cast<float2*>(Y + (16 * mr + g) * kLdA + 2 * t) = make_float2(c[0], c[1]);
+        *reinterpret_cast<float2*>(Y + (16 * mr + g + 8) * kLdA + 2 * t) = make_float2(c[2], c[3]);
     }
-    sync();
+    __syncwarp();
+    float c[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+    for (int mr = 0; mr < 2; ++mr)                     // X = -Tb Y
+        mma_tile_tf32<4>(sA + (32 + 16 * mr) * kLdA + 32, kLdA, Y, kLdA, c[mr], g, t);
+    __syncwarp();                                      // every lane has read Y and A_ba
+    {
+        const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+        *reinterpret_cast<float4*>(Y + lane * kLdA) = zero;
+        *reinterpret_cast<float4*>(Y + lane * kLdA + 4) = zero;
+    }
+#pragma unroll
+    for (int mr = 0; mr < 2; ++mr) {
+        float* dst = sA + (32 + 16 * mr) * kLdA + 8 * nb;
+        *reinterpret_cast<float2*>(dst + g * kLdA + 2 * t) = make_float2(-c[mr][0], -c[mr][1]);
+        *reinterpret_cast<float2*>(dst + (g + 8) * kLdA + 2 * t) = make_float2(-c[mr][2], -c[mr][3]);
+    }
 }
 
 // Lane 0 polls the mbarrier (bounded), the other lanes block at the warp barrier instead of
@@ -343,11 +363,11 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
     }
     tc_fence_before_sync();
     sync();
-    // Two jobs side by side: warps 0-1 invert the four diagonal 16x16 blocks of I + A (a serial
-    // forward substitution per column, 64 threads' worth of work), warps 2-7 scale the Q rows by
-    // scale * e^{b_r} in place (the Gram product has consumed Q): that is the Qg image.
+    // Two jobs side by side: warps 0-1 invert the two diagonal 32x32 blocks of I + A (serial
+    // forward substitutions and two small products each, all inside the warp), warps 2-7 scale
+    // the Q rows by scale * e^{b_r} in place (the Gram product has consumed Q): the Qg image.
     if (warp < 2) {
-        solve_diagonal_blocks(sA, tid);
+        solve_blocks_16_32(sA, warp, tid & 31, ci.len);
     } else {
 #pragma unroll 2
         for (int idx = tid - 64; idx < 1024; idx += kIntraThreads - 64) {      // 1024 16-byte pieces
@@ -364,16 +384,16 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
     }
     sync();
     if (tid == 0) {
-        // Qg is final: store it now; its shared memory is reused by the solve's merge levels.
-        // The scratch of those levels borrows the first Q half, which this bulk store is still
-        // reading: wait for the reads (not for the writes to land) before anyone goes on.
+        // Qg is final: store it now.  The T_w / T_u images are written over it next: wait for the
+        // bulk store's reads (not for its writes to land) meanwhile.
         bulk_store(rec + kRecQg, smem + kI_QK, 8192);
         bulk_store(rec + kRecQg + 8192, smem + kI_QK + 16384, 8192);
         bulk_commit();
         bulk_wait_read_all();
+    } else if (warp >= 4 && ci.len > 32) {
+        solve_merge_64(sA, warp - 4, tid & 31);        // (rows past the length are zero: nothing to do)
     }
     sync();
-    solve_merge_levels(sA, reinterpret_cast<float*>(smem + kI_Scr), tid, sync, ci.len);
 
     uint32_t tu_lo[2][4];    // T diag(beta) - bf16(T diag(beta)), parked until T_w is dead
     {   // T (fp32, row-major) -> bf16 B operands T diag(beta e^b), T diag(beta) (hi, lo)
