@@ -165,8 +165,11 @@ __device__ __forceinline__ void solve_blocks_16_32(float* sA, const int pr, cons
 }
 
 // Columns 8 nb .. 8 nb + 7 (nb = 0..3) of the 32x32 block (1, 0), by one warp, given the inverses
-// of the two diagonal 32x32 blocks.
-__device__ __forceinline__ void solve_merge_64(float* sA, const int nb, const int lane) {
+// of the two diagonal 32x32 blocks.  Called by four consecutive warps together: each reads all
+// of A_ba for its first product and writes its columns of the result over A_ba afterwards, so
+// the four meet at a barrier of their own (`bar_id`, 128 threads) in between.
+__device__ __forceinline__ void solve_merge_64(float* sA, const int nb, const int lane,
+                                               const int bar_id) {
     const int g = lane >> 2, t = lane & 3;
     float* Y = sA + 32 + 8 * nb;                       // rows 0-31 of the mirror block, zero on entry
 #pragma unroll
@@ -176,7 +179,7 @@ __device__ __forceinline__ void solve_merge_64(float* sA, const int nb, const in
         *reinterpret_cast<float2*>(Y + (16 * mr + g) * kLdA + 2 * t) = make_float2(c[0], c[1]);
         *reinterpret_cast<float2*>(Y + (16 * mr + g + 8) * kLdA + 2 * t) = make_float2(c[2], c[3]);
     }
-    __syncwarp();
+    asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");      // A_ba has been read by all four warps
     float c[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
     for (int mr = 0; mr < 2; ++mr)                     // X = -Tb Y
@@ -391,7 +394,9 @@ __device__ __forceinline__ bool intra_item(const TensorMaps& maps, const Prefill
         bulk_commit();
         bulk_wait_read_all();
     } else if (warp >= 4 && ci.len > 32) {
-        solve_merge_64(sA, warp - 4, tid & 31);        // (rows past the length are zero: nothing to do)
+        // (rows past the length are zero: nothing to do then).  Barrier ids 4.. are this routine's:
+        // one per group of 256 threads of the CTA.
+        solve_merge_64(sA, warp - 4, tid & 31, 4 + (static_cast<int>(threadIdx.x) >> 8));
     }
     sync();
 
