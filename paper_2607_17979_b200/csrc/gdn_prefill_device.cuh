@@ -543,20 +543,24 @@ constexpr uint32_t kS_Out = 2 * kStageBytes;   // o staging [64 tokens][128 dv] 
 constexpr uint32_t kT_D1 = 0, kT_Y = 64 /* two tiles of 64 */, kT_D4 = 192, kT_S = 320, kT_U = 384,
                    kT_Us = 416, kT_UsLo = 448;
 
-// bounded wait that also gives up as soon as another role has flagged an abort
-__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+// bounded wait that also gives up as soon as another role has flagged an abort.  `reason` is what a
+// wait that runs out writes into the flag: 1 = an error (reported as a timeout), 2 = give up
+// without an error (the caller's work is finished by a later launch).
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                              const int reason = 1) {
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((i & 255u) == 255u && *abort_flag) return false;
     }
-    if (*abort_flag == 0) *abort_flag = 1;      // keep an earlier, different reason
+    if (*abort_flag == 0) *abort_flag = reason;      // keep an earlier, different reason
     return false;
 }
 
 // Same, for a whole warp: lane 0 polls, every lane gets the verdict.
-__device__ __forceinline__ bool warp_wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool warp_wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                   const int reason = 1) {
     int ok = 1;
-    if ((threadIdx.x & 31) == 0) ok = wait_or_abort(bar, parity, abort_flag) ? 1 : 0;
+    if ((threadIdx.x & 31) == 0) ok = wait_or_abort(bar, parity, abort_flag, reason) ? 1 : 0;
     return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 

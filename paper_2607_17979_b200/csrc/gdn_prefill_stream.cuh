@@ -109,6 +109,12 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
     __shared__ uint64_t bar_full[2], bar_free_a[2], bar_free_b[2], bar_free_c[2], bar_y[2],
         bar_d1, bar_d4, bar_s, bar_u;
     __shared__ int abort_flag;
+    __shared__ uint32_t armed_chunks;     // chunks of the CTA's stream whose copies the loader has started
+    // kGated == 2 waits for records of a launch that may not be running beside this one: there no
+    // wait that runs out is an error, whichever role it happens in (the loader's own wait for a
+    // flag is the shortest, but the limits are counted in polls, not in time): the units this CTA
+    // has not finished are left to the last launch, which reports real failures.
+    constexpr int kWaitReason = kGated == 2 ? 2 : 1;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int half = (warp >> 2) & 1;                 // which half of the columns this thread owns
     const int dv = (warp & 3) * 32 + lane;            // TMEM lane = state row
@@ -143,6 +149,7 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
         mbar_init(&bar_s, kSEpiWarps + kSOutThreads / 32);
         mbar_init(&bar_u, kSEpiWarps);
         abort_flag = 0;
+        armed_chunks = 0;
         fence_barrier_init();
     }
     tc_fence_before_sync();
@@ -221,12 +228,13 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
                         // below; one here would also wait for this thread's copies in flight (3 %
                         // of a long sequence's run time).
                     }
-                    if (g >= 2 && !wait_or_abort(&bar_free_a[st], par_free, abortp)) { live = false; break; }
+                    if (g >= 2 && !wait_or_abort(&bar_free_a[st], par_free, abortp, kWaitReason)) { live = false; break; }
+                    armed_chunks = g + 1;
                     mbar_expect_tx(&bar_full[st], kRecBytes + 16384);
                     bulk_load(base + kS_Rec + kRecW, rec + kRecW, kRecP - kRecW, &bar_full[st]);
-                    if (g >= 2 && !wait_or_abort(&bar_free_b[st], par_free, abortp)) { live = false; break; }
+                    if (g >= 2 && !wait_or_abort(&bar_free_b[st], par_free, abortp, kWaitReason)) { live = false; break; }
                     bulk_load(base + kS_Rec + kRecU, rec + kRecU, kRecBytes - kRecU, &bar_full[st]);
-                    if (g >= 2 && !wait_or_abort(&bar_free_c[st], par_free, abortp)) { live = false; break; }
+                    if (g >= 2 && !wait_or_abort(&bar_free_c[st], par_free, abortp, kWaitReason)) { live = false; break; }
                     bulk_load(base + kS_Rec + kRecP, rec + kRecP, kRecU - kRecP, &bar_full[st]);
                     tma_load_2d(base + kS_K, &maps.k, u.hqk * kD, u.seq_t0 + j * kChunk, &bar_full[st]);
                     tma_load_2d(base + kS_K + 8192, &maps.k, u.hqk * kD + 64, u.seq_t0 + j * kChunk,
@@ -265,7 +273,7 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
                     const uint64_t w = st ? dW1 : dW0, qg = st ? dQ1 : dQ0, pp = st ? dP1 : dP0,
                                    kk = st ? dK1 : dK0;
                     const uint32_t tY = tmem + kT_Y + st * 64;
-                    if (!wait_or_abort(&bar_s, g & 1u, abortp)) {      // record landed, bf16 S and U~ in TMEM
+                    if (!wait_or_abort(&bar_s, g & 1u, abortp, kWaitReason)) {      // record landed, bf16 S and U~ in TMEM
                         live = false;
                         break;
                     }
@@ -291,7 +299,7 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
                     if (elect_one()) mma_ts_c<true>(tY, tS + 48, sdesc_advance(qg, 8192 + 64), id64);
                     if (elect_one()) mma_ts_c<true>(tY, tS + 56, sdesc_advance(qg, 8192 + 96), id64);
                     if (elect_one()) mma_commit(&bar_free_a[st]);                          // W and Qg have been read
-                    if (!wait_or_abort(&bar_u, g & 1u, abortp)) {         // U operands in TMEM
+                    if (!wait_or_abort(&bar_u, g & 1u, abortp, kWaitReason)) {         // U operands in TMEM
                         live = false;
                         break;
                     }
@@ -340,7 +348,7 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
         };
         bool ok = true;
         auto await = [&](uint64_t* bar, uint32_t parity) {   // bounded wait + tcgen05 fence
-            if (ok && !warp_wait_or_abort(bar, parity, abortp)) ok = false;
+            if (ok && !warp_wait_or_abort(bar, parity, abortp, kWaitReason)) ok = false;
             tc_fence_after_sync();
         };
         // Every warp runs every group barrier and hand-over below, also after a wait has failed
@@ -481,7 +489,7 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
         const int odv = q4 * 32 + lane;
         auto preload = [&](uint32_t gq) {       // chunk gq of the CTA's stream -> accumulator
             const int sq = gq & 1;
-            if (ok && !warp_wait_or_abort(&bar_full[sq], (gq >> 1) & 1u, abortp)) ok = false;
+            if (ok && !warp_wait_or_abort(&bar_full[sq], (gq >> 1) & 1u, abortp, kWaitReason)) ok = false;
             if (ok) {
                 const float4* sU = reinterpret_cast<const float4*>(smem + sq * kStageBytes + kS_Rec + kRecU);
 #pragma unroll
@@ -518,7 +526,7 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
 #pragma unroll 1
                 for (int k = preloaded ? 1 : 0; k < 2; ++k) {
                     if (k == 1) {
-                        if (ok && !warp_wait_or_abort(&bar_u, g & 1u, abortp)) ok = false;
+                        if (ok && !warp_wait_or_abort(&bar_u, g & 1u, abortp, kWaitReason)) ok = false;
                         tc_fence_after_sync();
                         if (!ahead) break;
                     }
@@ -526,7 +534,7 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
                 }
                 preloaded = ahead;
                 // every warp runs both group barriers of every chunk, also after a failed wait
-                if (ok && !warp_wait_or_abort(&bar_y[buf], (g >> 1) & 1u, abortp)) ok = false;
+                if (ok && !warp_wait_or_abort(&bar_y[buf], (g >> 1) & 1u, abortp, kWaitReason)) ok = false;
                 tc_fence_after_sync();
                 // The Y tile (lanes = dv, columns = tokens) is read as accumulator fragments, rounded
                 // in pairs and stored transposed, 8 dv of one token per 16 bytes, into a [token][dv]
@@ -579,9 +587,13 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
     __syncthreads();
     if (abort_flag != 0 && warp == kSIssueWarp && lane == 0) {
         if (abort_flag == 1) report(p.dev_status, kDevTimeout);     // 2: a record not produced yet, no error
-        // let copies already in flight land before the CTA's shared memory goes away
-        mbar_wait(&bar_full[0], 0, 1u << 12);
-        mbar_wait(&bar_full[1], 0, 1u << 12);
+        // let copies already in flight land before the CTA's shared memory goes away: the last two
+        // chunks the loader started, each on its stage's barrier at that chunk's own parity
+        const uint32_t armed = *reinterpret_cast<volatile uint32_t*>(&armed_chunks);
+        for (uint32_t back = 1; back <= 2 && back <= armed; ++back) {
+            const uint32_t gq = armed - back;
+            mbar_wait(&bar_full[gq & 1], (gq >> 1) & 1u, 1u << 12);
+        }
     }
 }
 

@@ -7,6 +7,7 @@ GDN tables, on seeded synthetic inputs.  Prints one JSON object per shape and a 
     python sweep.py --lens 512,1024,2048,4096 --route overlap --split-permille 1000
     python sweep.py --decode-multi 64x4                # one multi-token shape
     python sweep.py --decode 256 --slots 512 --reps 40 # one decode shape
+    python sweep.py --gate 8192 | --transpose 64       # the gate helper / the tile transpose
 
 Each shape's call is captured `GRAPH_CALLS` times into one CUDA graph, and the graph is replayed
 and timed with CUDA events: the number is device time per call including kernel launch gaps but
@@ -100,6 +101,23 @@ def _decode_row(B, reps, slots=None, host=False):
     return row
 
 
+def _gate_row(T, reps):
+    d = I.gate_inputs(T, 32, seed=I.BASE_SEED + T)
+    a, b = _bf16(d["a"]), _bf16(d["b"])
+    A_log, dt_bias = _dev(d["A_log"]), _dev(d["dt_bias"])
+    g = torch.empty((T, 32), dtype=torch.float32, device="cuda")
+    beta = torch.empty_like(g)
+    us = _time(lambda: api.gdn_gate(a, b, A_log, dt_bias, g, beta), reps)
+    return {"op": "gate", "T": T, "Hv": 32, "us": us}
+
+
+def _transpose_row(n, reps):
+    pool = torch.randn((n, 32, 128, 128), dtype=torch.float32, device="cuda")
+    us = _time(lambda: api.gdn_state_transpose(pool), reps)
+    return {"op": "state_transpose", "slots": n, "Hv": 32, "us": us,
+            "GBps": 2 * n * 32 * 65536 / us / 1e3}
+
+
 def _prefill_row(lens, route, reps, split_permille=-1, host=False):
     p = I.prefill_inputs(lens, 16, 32, 128, seed=I.BASE_SEED + sum(lens), init="zero")
     t = {n: _bf16(p[n]) for n in "qkv"}
@@ -160,11 +178,20 @@ def main():
                     "BxL (both state orientations)")
     ap.add_argument("--decode", type=int, default=0, help="time one decode batch size only")
     ap.add_argument("--slots", type=int, default=0, help="pool slots for --decode (default: B)")
+    ap.add_argument("--gate", type=int, default=0, help="time the gate helper on this many tokens only")
+    ap.add_argument("--transpose", type=int, default=0, help="time the in-place tile transpose on "
+                    "this many slots only")
     args = ap.parse_args()
     if args.decode_multi:
         B, _, L = args.decode_multi.partition("x")
         for r in _multi_rows(int(B), int(L), args.reps):
             print(json.dumps(r))
+        return
+    if args.gate:
+        print(json.dumps(_gate_row(args.gate, args.reps)))
+        return
+    if args.transpose:
+        print(json.dumps(_transpose_row(args.transpose, args.reps)))
         return
     if args.decode:
         print(json.dumps(_decode_row(args.decode, args.reps, slots=args.slots or None, host=True)))
