@@ -207,12 +207,13 @@ int gdn_prefill(const void* q, const void* k, const void* v,
  * chunked variants (gdn_prefill_fused for a few long sequence-heads,
  * gdn_prefill_overlap when max_seqlen_hint tells of chains of at least 40
  * chunks and the sequence-heads number between a third and half of the SMs,
- * gdn_prefill_stream for chains longer than two chunks, more
- * sequence-heads than SMs or at most 16 sequences, else gdn_prefill_chunked).  Each route can also be called directly; arguments
- * are gdn_prefill's.  gdn_prefill_route answers which one gdn_prefill would take
- * (host-only arithmetic on the shapes; sm_count and cooperative_launch describe
- * the device, gdn_prefill itself queries them): one of GDN_ROUTE_*, or
- * GDN_ROUTE_NONE for an empty batch.
+ * gdn_prefill_stream for everything else).  Each route can also be called
+ * directly; arguments are gdn_prefill's.  gdn_prefill_chunked is the three
+ * launches under their older name: it runs gdn_prefill_stream.
+ * gdn_prefill_route answers which one gdn_prefill would take (host-only
+ * arithmetic on the shapes; sm_count and cooperative_launch describe the
+ * device, gdn_prefill itself queries them): one of GDN_ROUTE_* (never
+ * GDN_ROUTE_CHUNKED any more), or GDN_ROUTE_NONE for an empty batch.
  */
 #define GDN_RECURRENT_MAX_SEQLEN 16
 #define GDN_ROUTE_NONE      0

@@ -265,14 +265,9 @@ int gdn_prefill_route(int32_t T, int32_t N, int32_t max_seqlen_hint, int32_t Hv,
     // next, and batches of equal chains lose up to 7 %: those stay with the persistent pass.
     if (max_seqlen_hint > 0 && units <= sm_count / 2 && longest >= 40 * gdn::kChunk)
         return GDN_ROUTE_OVERLAP;
-    // The persistent state pass has the shorter chunk step (its loader, issuer, chain and output
-    // warps are separate) and does not pay a CTA start, a pipeline fill and a drain per unit:
-    // measured faster whenever a chain is longer than two chunks or there are more units than
-    // SMs, and for every batch of few sequences (no table-building launch then).  What is left,
-    // many short sequences of few heads, goes to the plain pass with its cheaper table-building
-    // launch, ahead there by a microsecond or two.
-    if (longest > 2 * gdn::kChunk || units > sm_count || N <= gdn::kInlineTableSeqs) return GDN_ROUTE_STREAM;
-    return GDN_ROUTE_CHUNKED;
+    // Everything else: the three launches (table kernel, or none for small batches; the intra-chunk
+    // kernel over all items; the persistent state pass).
+    return GDN_ROUTE_STREAM;
 }
 
 int gdn_prefill(const void* q, const void* k, const void* v, const float* g, const float* beta,

@@ -113,13 +113,12 @@ def test_prefill_routing_rules_are_pure_host_arithmetic():
     assert r(32768, 1, 0, 32) == "fused" and r(32768, 1, 0, 32, 148, False) == "stream"
     assert r(1025, 1, 0, 32) == "fused" and r(1024, 1, 0, 32) == "stream"
     assert r(32768, 1, 0, 49) == "fused" and r(32768, 1, 0, 50) == "stream"       # 148 // 3 = 49 units
-    # a chain longer than two chunks, more units than SMs, or at most 16 sequences: the persistent
-    # state pass
+    # everything else that is chunked: the three launches with the persistent state pass
     assert r(7680, 4, 0, 32) == "stream" and r(129, 1, 0, 32) == "stream"
     assert r(128, 1, 0, 32) == "stream" and r(400, 4, 100, 32) == "stream"
-    assert r(1600, 16, 100, 4) == "stream" and r(1700, 17, 100, 4) == "chunked"
-    assert r(8192, 128, 64, 32) == "stream" and r(296, 37, 8, 4) != "stream"        # 4096 / 148 units
-    assert r(1184, 37, 32, 4) == "chunked" and r(1216, 38, 32, 4) == "stream"       # 148 / 152 units
+    assert r(1600, 16, 100, 4) == "stream" and r(1700, 17, 100, 4) == "stream"
+    assert r(8192, 128, 64, 32) == "stream" and r(296, 37, 8, 4) == "recurrent"
+    assert r(1184, 37, 32, 4) == "stream" and r(1216, 38, 32, 4) == "stream"
     # the caller says how long the longest sequence is, chains of at least 40 chunks, more units
     # than the cooperative launch takes and at most half as many as SMs: the two-part production
     assert r(8192, 2, 4096, 32) == "overlap" and r(4000, 2, 3000, 32) == "overlap"
