@@ -522,7 +522,7 @@ __device__ __forceinline__ void state_stream_role(const TensorMaps& maps, const 
                 // k = 1: once the chain warps have read U of this chunk the accumulator is free for
                 // the next chunk's U~ (when the next chunk is known without looking past a skipped
                 // unit), which is then in place long before the chain warps hand the state over.
-                const bool ahead = j + 1 < u.nc || (unit + n_ctas < total_units && !nxt.skip);
+                const bool ahead = j + 1 < u.nc || (unit + n_ctas < total_units && !nxt.skip && !nxt.done);
 #pragma unroll 1
                 for (int k = preloaded ? 1 : 0; k < 2; ++k) {
                     if (k == 1) {
